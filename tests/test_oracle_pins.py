@@ -1,0 +1,360 @@
+"""Pins for the CPU oracle: closed forms, invariants, library routines and brute force.
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped term, a wrong
+sign or index, a transposed operand, a wrong rounding rule) makes it fail.  None of them
+needs a GPU and none calls the CUDA path.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import qcfg_workloads as wl
+from oracle import qcfg_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+BITS = list(range(2, 9))
+
+
+def _golden(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+# ----------------------------------------------------------------------- absmax and scales
+
+@pytest.mark.parametrize("b", BITS)
+def test_absmax_element_maps_to_qmax(b):
+    rng = np.random.default_rng(b)
+    for _ in range(200):
+        x = (rng.standard_normal(257) * 10.0 ** rng.uniform(-6, 6)).astype(np.float32)
+        A = orc.absmax(x)
+        s, inv = orc.scales_from_absmax(A, b)
+        q = orc.quantize(x, inv, b)
+        i = int(np.argmax(np.abs(x)))
+        assert abs(int(q[i])) == orc.qmax(b)
+        assert int(np.sign(q[i])) == int(np.sign(x[i]))
+        assert abs(float(s) * float(inv) - 1.0) < 3 * 2.0 ** -23
+
+
+def test_absmax_is_absolute_and_per_row():
+    x = np.array([[1.0, -7.0, 3.0], [-0.5, 0.25, 0.125]], dtype=np.float32)
+    assert orc.absmax(x) == np.float32(7.0)            # a signed max would give 3
+    np.testing.assert_array_equal(orc.absmax(x, orc.PER_ROW), np.array([7.0, 0.5], np.float32))
+
+
+def test_zero_tensor_is_defined():
+    x = np.zeros((3, 4), np.float32)
+    s, inv = orc.scales_from_absmax(orc.absmax(x), 4)
+    assert s == 1 and inv == 1
+    assert not orc.quantize(x, inv, 4).any()
+    sse, amax = orc.quant_error_sweep([x])
+    assert not sse.any() and amax[0] == 0
+    assert orc.e_qe(0.0, 12, 0.0) == 0.0
+
+
+# ----------------------------------------------------------------------- quantizer (Eq. 1)
+
+@pytest.mark.parametrize("b", BITS)
+def test_levels_monotone_odd(b):
+    rng = np.random.default_rng(100 + b)
+    x = np.sort(rng.standard_normal(20000).astype(np.float32) * 3)
+    _, inv = orc.scales_from_absmax(orc.absmax(x), b)
+    q = orc.quantize(x, inv, b).astype(np.int32)
+    assert len(np.unique(q)) <= 2 ** b - 1
+    assert q.min() >= -orc.qmax(b) and q.max() <= orc.qmax(b)
+    assert np.all(np.diff(q) >= 0)
+    np.testing.assert_array_equal(orc.quantize(-x, inv, b).astype(np.int32), -q)
+
+
+@pytest.mark.parametrize("b", BITS)
+def test_idempotent_all_codes(b):
+    rng = np.random.default_rng(7)
+    codes = np.arange(-orc.qmax(b), orc.qmax(b) + 1, dtype=np.int8)
+    for _ in range(300):
+        A = np.float32(10.0 ** rng.uniform(-8, 8))
+        s, inv = orc.scales_from_absmax(A, b)
+        np.testing.assert_array_equal(orc.quantize(orc.dequantize(codes, s), inv, b), codes)
+
+
+@pytest.mark.parametrize("b", [3, 4, 8])
+def test_ties_round_to_even_and_clip(b):
+    qm = orc.qmax(b)
+    A = np.float32(qm * 0.25)                 # scale = 0.25 and inv_scale = 4 exactly
+    s, inv = orc.scales_from_absmax(A, b)
+    assert s == np.float32(0.25) and inv == np.float32(4.0)
+    k = np.arange(-qm, qm, dtype=np.float32)
+    x = (k + np.float32(0.5)) * np.float32(0.25)      # exact ties
+    q = orc.quantize(x, inv, b).astype(np.int32)
+    assert np.all(q % 2 == 0)
+    assert np.all(np.abs(q - (k + 0.5)) == 0.5)
+    big = np.array([10 * A, -10 * A], np.float32)     # beyond the calibrated range
+    np.testing.assert_array_equal(orc.quantize(big, inv, b), np.array([qm, -qm], np.int8))
+
+
+@pytest.mark.parametrize("b", BITS)
+def test_fake_quant_matches_library_on_exact_scales(b):
+    """With a power-of-two scale both the oracle and torch's fake-quantize are exact."""
+    rng = np.random.default_rng(b)
+    qm = orc.qmax(b)
+    rows = np.array([qm * 2.0 ** -3, qm * 2.0 ** -5, qm * 2.0 ** 1], np.float32)
+    x = rng.uniform(-1, 1, size=(3, 500)).astype(np.float32) * rows[:, None]
+    x[:, 0] = rows                                      # the row maxima
+    got = orc.fake_quant(x, b, orc.PER_ROW)
+    scale = torch.tensor(rows / qm)
+    want = torch.fake_quantize_per_channel_affine(torch.from_numpy(x), scale,
+                                                  torch.zeros(3, dtype=torch.int32), 0, -qm, qm)
+    np.testing.assert_array_equal(got, want.numpy())
+
+
+def test_bf16_round_matches_library_everywhere():
+    hi = np.arange(2 ** 16, dtype=np.uint32) << 16
+    lows = np.array([0x0000, 0x0001, 0x7FFF, 0x8000, 0x8001, 0xFFFF], np.uint32)
+    u = (hi[:, None] | lows[None, :]).reshape(-1)
+    x = u.view(np.float32)
+    finite = np.isfinite(x)
+    got = orc.bf16_round(x[finite])
+    want = torch.from_numpy(x[finite].copy()).to(torch.bfloat16).to(torch.float32).numpy()
+    ok = np.isfinite(want)                              # rounding up to inf is out of scope
+    np.testing.assert_array_equal(got[ok].view(np.uint32), want[ok].view(np.uint32))
+
+
+# ----------------------------------------------------------------------- E_QE (Eq. 2)
+
+def test_uniform_closed_form():
+    n = 1 << 20
+    A = 3.0
+    x = (np.linspace(-A, A, n, dtype=np.float64)).astype(np.float32)[None, :]
+    sse, amax = orc.quant_error_sweep([x], orc.PER_TENSOR)
+    for b, want in _golden("uniform_eqe.txt"):
+        got = orc.e_qe(sse[0, int(b) - 2], n, amax[0])
+        assert got == pytest.approx(float(want), rel=2e-3), b
+
+
+def test_sse_bound_decreasing_and_zero_on_grid():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((37, 301)).astype(np.float32) * rng.uniform(0.1, 10, (37, 1)).astype(np.float32)
+    sse, amax = orc.quant_error_sweep([x], orc.PER_ROW)
+    assert np.all(np.diff(sse[0]) < 0)
+    for j, b in enumerate(BITS):
+        s, _ = orc.scales_from_absmax(orc.absmax(x, orc.PER_ROW), b)
+        bound = float(np.sum(x.shape[1] * s.astype(np.float64) ** 2 / 4))
+        assert sse[0, j] <= bound * (1 + 1e-6)
+        xg = orc.fake_quant(x, b, orc.PER_ROW)            # already on the b-bit grid
+        assert orc.quant_error_sse(xg, b, orc.PER_ROW) <= 1e-12 * float(np.sum(xg.astype(np.float64) ** 2))
+
+
+def test_sse_brute_force_small():
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((3, 5)).astype(np.float32)
+    sse, amax = orc.quant_error_sweep([x], orc.PER_ROW)
+    for j, b in enumerate(BITS):
+        qm = 2 ** (b - 1) - 1
+        tot = 0.0
+        for r in range(3):
+            A = max(abs(float(v)) for v in x[r])
+            for v in x[r]:
+                v = float(v)
+                code = max(-qm, min(qm, round(v * qm / A)))      # python round: half-even
+                tot += (v - code * A / qm) ** 2
+        assert sse[0, j] == pytest.approx(tot, rel=1e-5)
+    assert float(amax[0]) == max(abs(float(v)) for v in x.reshape(-1))
+
+
+def test_per_row_reduces_to_per_tensor_and_eqe_normalisation():
+    rng = np.random.default_rng(5)
+    x = rng.uniform(-1, 1, (8, 64)).astype(np.float32)
+    x[:, 3] = np.float32(2.0) * np.where(np.arange(8) % 2, 1, -1)   # every row has absmax 2
+    for b in (2, 5, 8):
+        assert orc.quant_error_sse(x, b, orc.PER_ROW) == orc.quant_error_sse(x, b, orc.PER_TENSOR)
+    sse = orc.quant_error_sse(x, 4, orc.PER_TENSOR)
+    e = orc.e_qe(sse, x.size, 2.0)
+    assert e == pytest.approx(math.sqrt(sse / x.size) / 2.0, rel=1e-12)
+    # scale invariance of Eq. 2 under power-of-two rescaling of the tensor (exact in fp32)
+    sse4 = orc.quant_error_sse(x * np.float32(4), 4, orc.PER_TENSOR)
+    assert orc.e_qe(sse4, x.size, 8.0) == pytest.approx(e, rel=1e-12)
+
+
+def test_ranking_stable_ascending():
+    r = orc.ranking([0.3, 0.1, 0.3, 0.05, 0.1])
+    np.testing.assert_array_equal(r, [3, 1, 4, 0, 2])
+
+
+# ----------------------------------------------------------------------- integer GEMM
+
+def test_int_gemm_brute_force_and_library():
+    rng = np.random.default_rng(2)
+    qx = rng.integers(-127, 128, (5, 19), dtype=np.int8)
+    qw = rng.integers(-127, 128, (7, 19), dtype=np.int8)
+    acc = orc.int_gemm(qx, qw)
+    assert acc.dtype == np.int32 and acc.shape == (5, 7)
+    for m in range(5):
+        for n in range(7):
+            assert int(acc[m, n]) == sum(int(qx[m, k]) * int(qw[n, k]) for k in range(19))
+    qx = rng.integers(-127, 128, (33, 300), dtype=np.int8)
+    qw = rng.integers(-127, 128, (21, 300), dtype=np.int8)
+    np.testing.assert_array_equal(orc.int_gemm(qx, qw), qx.astype(np.int64) @ qw.astype(np.int64).T)
+
+
+def test_int_gemm_worst_case_magnitude():
+    K = 4608
+    qx = np.full((2, K), 127, np.int8)
+    qw = np.stack([np.full(K, 127, np.int8), np.full(K, -127, np.int8)])
+    acc = orc.int_gemm(qx, qw)
+    assert acc[0, 0] == K * 127 * 127 and acc[1, 1] == -K * 127 * 127
+
+
+# ----------------------------------------------------------------------- epilogue
+
+def test_gelu_identity_limits_and_library():
+    y = np.concatenate([np.linspace(-12, 12, 4001), [0.0, 50.0, -50.0, 1e4, -1e4]]).astype(np.float32)
+    g = orc.gelu_tanh(y)
+    assert np.all(np.isfinite(g))
+    y64 = y.astype(np.float64)
+    ref = 0.5 * y64 * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (y64 + 0.044715 * y64 ** 3)))
+    np.testing.assert_allclose(g, ref, rtol=1e-6, atol=1e-12)
+    lib = torch.nn.functional.gelu(torch.from_numpy(y64), approximate="tanh").numpy()
+    np.testing.assert_allclose(g, lib, rtol=1e-6, atol=1e-12)
+    assert orc.gelu_tanh(np.float32(0)) == 0
+    assert orc.gelu_tanh(np.float32(50)) == np.float32(50)
+    assert orc.gelu_tanh(np.float32(-50)) == 0
+
+
+def test_dequant_and_relu_exact():
+    acc = np.array([[3, -5], [2 ** 24 + 1, -7]], np.int32)
+    sw = np.array([0.5, 0.25], np.float32)
+    y = orc.dequant_output(acc, np.float32(2.0), sw)
+    np.testing.assert_array_equal(y, np.array([[3.0, -2.5], [float(np.float32(2 ** 24 + 1)), -3.5]], np.float32))
+    np.testing.assert_array_equal(orc.activation(y, orc.ACT_RELU)[:, 1], [0, 0])
+
+
+# ----------------------------------------------------------------------- layers and chains
+
+def test_bf16_layer_matches_library_matmul():
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((40, 96)).astype(np.float32)
+    w = rng.standard_normal((24, 96)).astype(np.float32)
+    got = orc.bf16_gemm(x, w)
+    xb = torch.from_numpy(x).to(torch.bfloat16).double()
+    wb = torch.from_numpy(w).to(torch.bfloat16).double()
+    np.testing.assert_allclose(got, (xb @ wb.T).numpy(), rtol=1e-6, atol=1e-6)
+    full = x.astype(np.float64) @ w.astype(np.float64).T
+    assert np.linalg.norm(got - full) / np.linalg.norm(full) < 1e-2
+
+
+@pytest.mark.parametrize("k,stride,pad", [(1, 1, 0), (1, 2, 0), (3, 1, 1), (3, 2, 1), (7, 2, 3)])
+def test_conv_as_im2col_matches_library(k, stride, pad):
+    rng = np.random.default_rng(k * 10 + stride)
+    B, H, W, C, N = 2, 13, 11, 5, 6
+    x = orc.bf16_round(rng.standard_normal((B, H, W, C)).astype(np.float32))
+    w = orc.bf16_round(rng.standard_normal((N, k, k, C)).astype(np.float32))     # OHWI
+    lay = wl.Layer("c", N, k * k * C, kh=k, kw=k, stride=stride, pad=pad, in_h=H, in_w=W, in_c=C)
+    y = orc.bf16_gemm(orc.gemm_rows(lay, x), w.reshape(N, -1))
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).double().permute(0, 3, 1, 2),
+                                     torch.from_numpy(w).double().permute(0, 3, 1, 2),
+                                     stride=stride, padding=pad)
+    ref = ref.permute(0, 2, 3, 1).reshape(-1, N).numpy()
+    assert y.shape == (B * lay.out_h * lay.out_w, N)
+    np.testing.assert_allclose(y, ref, rtol=1e-5, atol=1e-5)
+
+
+def test_pools_match_library():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((2, 9, 12, 3)).astype(np.float32)
+    t = torch.from_numpy(x).permute(0, 3, 1, 2)
+    mp = torch.nn.functional.max_pool2d(t, 3, 2, 1).permute(0, 2, 3, 1).numpy()
+    np.testing.assert_array_equal(orc.maxpool3s2(x), mp)
+    ap = t.double().mean(dim=(2, 3)).float().numpy()
+    np.testing.assert_allclose(orc.global_avgpool(x), ap, rtol=1e-6)
+
+
+def test_quantized_layer_tracks_float_layer():
+    """A quantized layer approximates the float product with an error that shrinks with b;
+    a transposed operand, a missing scale or a wrong dequantization would break this."""
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((64, 128)).astype(np.float32)
+    w = (rng.standard_normal((48, 128)) * 0.05).astype(np.float32)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    lay = wl.Layer("l", 48, 128)
+    errs = []
+    for b in (4, 6, 8):
+        y = orc.layer_forward(lay, w, x, b, orc.absmax(x), orc.absmax(w, orc.PER_ROW))
+        errs.append(np.linalg.norm(y - ref) / np.linalg.norm(ref))
+    assert errs[0] > errs[1] > errs[2]
+    assert errs[2] < 0.02 and errs[0] < 0.35
+
+
+def test_chain_all16_equals_calibration_forward_and_taps_consistent():
+    w = wl.bert_stack(seed=5, m=24, hidden=32, ffn=64, n_blocks=2)
+    act_amax, w_amax = orc.calibrate_model(w.layers, w.weights, w.x)
+    outs16 = orc.eval_config(w.layers, w.weights, [16] * 12, w.x, act_amax, w_amax)
+    # the calibrated activation maxima are the maxima of the 16-bit forward's layer inputs
+    for l, lay in enumerate(w.layers):
+        src = w.x if lay.src < 0 else outs16[lay.src]
+        assert act_amax[l] == np.max(np.abs(src))
+    outs, taps = orc.eval_config(w.layers, w.weights, w.bits, w.x, act_amax, w_amax, want_taps=True)
+    for l, lay in enumerate(w.layers):
+        if w.bits[l] == 16:
+            continue
+        t = taps[l]
+        src = w.x if lay.src < 0 else outs[lay.src]
+        np.testing.assert_array_equal(t["a"], src)
+        y, t2 = orc.eval_layer_teacher_forced(lay, w.weights[l], src, int(w.bits[l]), act_amax[l], w_amax[l])
+        np.testing.assert_array_equal(y, outs[l])
+        np.testing.assert_array_equal(t2["acc"], t["acc"])
+    # dependence structure of the stand-in graph: V feeds O, Q/K feed nobody
+    assert w.layers[3].src == 2 and w.layers[4].src == 3 and w.layers[6].src == 5
+    assert all(l.src not in (0, 1) for l in w.layers)
+
+
+def test_resnet_chain_small_runs_and_residual_is_used():
+    w = wl.resnet50(seed=3, batch=1, in_hw=32, width=8, n_classes=10, blocks=(1, 1, 1, 1))
+    act_amax, w_amax = orc.calibrate_model(w.layers, w.weights, w.x)
+    outs = orc.eval_config(w.layers, w.weights, w.bits, w.x, act_amax, w_amax)
+    assert outs[-1].shape == (1, 10)
+    assert all(np.all(np.isfinite(o)) for o in outs)
+    c = next(i for i, l in enumerate(w.layers) if l.residual_from >= 0)
+    lay = w.layers[c]
+    xin = orc.layer_input(w.layers, c, w.x, outs)
+    no_res = orc.layer_forward(lay, w.weights[c], xin, int(w.bits[c]), act_amax[c], w_amax[c])
+    assert not np.array_equal(no_res, outs[c])
+    assert np.all(outs[c] >= 0)
+
+
+# ----------------------------------------------------------------------- tables and sequences
+
+def test_layer_tables_match_table1_sizes():
+    res = wl.resnet50_layers()
+    bert = wl.bert_layers(1024, 4096, 24)
+    assert len(res) == 54 and wl.param_count(res) == 25_502_912
+    assert len(bert) == 144 and wl.param_count(bert) == 301_989_888
+    assert wl.param_count(wl.bert_layers(768, 3072, 12)) == 84_934_656
+    tables = {"resnet50": res, "bert": bert}
+    for model, b, mb in _golden("table1_sizes.txt"):
+        L = tables[model]
+        assert wl.size_mb(L, [int(b)] * len(L)) == pytest.approx(float(mb), abs=0.0075)
+
+
+def test_search_sequences_follow_the_algorithms():
+    n = 72
+    rank = np.random.default_rng(0).permutation(n)
+    acc = np.random.default_rng(1).random(n) < 0.5
+    seq = wl.greedy_sequence(rank, acc)
+    assert len(seq) == n                                   # one evaluation per layer per bit width
+    for i, cfg in enumerate(seq):
+        assert cfg[rank[i]] == 4
+        kept = [rank[j] for j in range(i) if acc[j]]
+        dropped = [rank[j] for j in range(i) if not acc[j]]
+        assert np.all(cfg[kept] == 4) and np.all(cfg[dropped] == 8)
+    rank = np.arange(144)
+    seq = wl.bisection_sequence(rank, [True, False, True, True, False, False, True, True], 108, 8)
+    counts = [int(np.sum(c == 4)) for c in seq]
+    assert counts[:4] == [54, 81, 68, 74]                  # +27, -(27//2), +(13//2): floor halving
+    assert all(int(np.sum(c == 16)) == 36 for c in seq)
+    assert len(seq) <= 3 * math.ceil(math.log2(144)) + 3
