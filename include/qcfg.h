@@ -1,0 +1,182 @@
+/*
+ * qcfg -- evaluation of candidate bit configurations and the quantization-error
+ * sensitivity sweep for sensitivity-guided mixed-precision post-training quantization
+ * (Schaefer et al., "Mixed Precision Post Training Quantization of Neural Networks with
+ * Sensitivity Guided Search"), for one NVIDIA B200 (sm_100a).
+ *
+ * Conventions shared by every entry point
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; the library never
+ *     frees or reallocates them.  Pointers without that suffix are HOST pointers.
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued asynchronously on it
+ *     unless stated otherwise.
+ *   - Every call returns a status code (QCFG_OK = 0), never throws, aborts or prints.
+ *     On a non-OK return no output has been written.  Errors detected on the device
+ *     (a bounded wait that gave up, a non-finite calibration maximum) surface from
+ *     qcfg_sync_status().
+ *   - Matrices are row-major.  A weight is [n_out x k_in] fp32, row = output channel; for
+ *     a convolution k_in = kh*kw*in_c in (kh, kw, cin) order (OHWI).  An activation is
+ *     [m x k] fp32 (for convolutions: NHWC, i.e. [batch*h*w x c]).
+ *   - Bit widths: 2..8 are symmetric signed integer grids with qmax = 2^(b-1)-1 (codes held
+ *     in int8); 16 is bfloat16 operands with fp32 accumulation.
+ *   - There is no CPU fallback: without an sm_100 device qcfg_create() fails.
+ */
+#ifndef QCFG_H_
+#define QCFG_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qcfg_ctx qcfg_ctx;     /* device, workspace, tensor-map encoder, error word */
+typedef struct qcfg_model qcfg_model; /* layer table, weight-code cache, calibration tables  */
+
+enum {
+  QCFG_OK = 0,
+  QCFG_EINVAL = 1,     /* null pointer, bad enum, negative size                     */
+  QCFG_EBITS = 2,      /* bit width outside {2..8, 16} (or outside 2..8 where stated) */
+  QCFG_ESHAPE = 3,     /* inconsistent shapes / layer graph                         */
+  QCFG_EALIGN = 4,     /* pointer or leading dimension alignment                    */
+  QCFG_ENOMEM = 5,     /* device allocation failed                                  */
+  QCFG_ENONFINITE = 6, /* a calibration maximum is NaN or Inf                       */
+  QCFG_EARCH = 7,      /* device is not sm_100                                      */
+  QCFG_ECUDA = 8,      /* a CUDA runtime/driver call failed; see qcfg_last_error    */
+  QCFG_ETIMEOUT = 9,   /* a bounded device-side wait gave up                        */
+  QCFG_EUNIMPL = 10,   /* feature not available in this build                       */
+  QCFG_ESTATE = 11     /* call order (e.g. evaluation before calibration)           */
+};
+enum { QCFG_PER_TENSOR = 0, QCFG_PER_ROW = 1 };
+enum { QCFG_ACT_NONE = 0, QCFG_ACT_RELU = 1, QCFG_ACT_GELU_TANH = 2 };
+enum { QCFG_POOL_NONE = 0, QCFG_POOL_MAX3S2 = 1, QCFG_POOL_GLOBAL_AVG = 2 };
+
+/* One "tensor" of the bit configuration: a linear or convolution layer whose weight and
+ * input activation share one bit width (Algorithms 1 and 2 index the configuration by
+ * layer; Table 1: "same bit-precision for all their weights and activations").           */
+typedef struct qcfg_layer {
+  const float* w_dev;    /* [n_out][k_in] fp32, borrowed for the model's lifetime          */
+  int64_t n_out, k_in;
+  int32_t src;           /* -1 = external input, else index of the producing layer (< own) */
+  int32_t src_col0;      /* first column of the producer's output that is read             */
+  int32_t act;           /* QCFG_ACT_*, applied to this layer's output after the residual  */
+  int32_t kh, kw, stride, pad;  /* convolution geometry; all 0 for a linear layer          */
+  int32_t in_h, in_w, in_c;     /* input size after pool_before (conv only)                */
+  int32_t pool_before;          /* QCFG_POOL_*, applied in fp32 to the source              */
+  int32_t src_h, src_w;         /* spatial size of the source before pool_before           */
+  int32_t residual_from;        /* -1, or a layer whose fp32 output is added before act    */
+} qcfg_layer;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device`.  QCFG_EARCH if it is not compute capability
+ * 10.x, QCFG_ECUDA if the runtime fails.  The context allocates a small device error word
+ * and grows scratch buffers on demand (cudaMalloc on first use of a larger size).        */
+int qcfg_create(qcfg_ctx** out, int device);
+int qcfg_destroy(qcfg_ctx* ctx);
+
+/* Synchronises `stream`, then returns and clears the device error word:
+ * QCFG_OK, QCFG_ETIMEOUT, QCFG_ENONFINITE or QCFG_ECUDA.                                  */
+int qcfg_sync_status(qcfg_ctx* ctx, void* stream);
+/* Library-owned, NUL-terminated description of the last non-OK status of this context.   */
+const char* qcfg_last_error(qcfg_ctx* ctx);
+/* Number of kernels this context has launched since creation (for accounting).            */
+int64_t qcfg_launch_count(qcfg_ctx* ctx);
+
+/* ---- tensor-level steps --------------------------------------------------------------- */
+
+/* Max calibration (Section 3.1: the maximum value of each tensor; absolute value as in
+ * Eq. 2).  x_dev is [rows x cols] fp32 with leading dimension ld (elements).
+ * QCFG_PER_TENSOR writes 1 float, QCFG_PER_ROW writes `rows` floats to absmax_dev.  A NaN
+ * or Inf input yields a non-finite maximum.                                               */
+int qcfg_calibrate(qcfg_ctx* ctx, const float* x_dev, int64_t rows, int64_t cols, int64_t ld,
+                   int granularity, float* absmax_dev, void* stream);
+
+/* The two scales of Eq. 1 for a b-bit grid, b in 2..8: scale = A/qmax (applied after the
+ * rounding, the paper's 2^-(b-1)*gamma) and inv_scale = qmax/A (applied before it, the
+ * paper's alpha*2^(b-1)); one IEEE fp32 division each; A == 0 gives 1 and 1.  Either output
+ * may be NULL.                                                                             */
+int qcfg_scales_from_absmax(qcfg_ctx* ctx, const float* absmax_dev, int64_t n, int bits,
+                            float* scale_dev, float* inv_scale_dev, void* stream);
+
+/* Codes of Eq. 1: q = clamp(round_half_even(x * inv_scale), -qmax, +qmax) as int8 for bits
+ * in 2..8; for bits == 16 the output is bfloat16 (round to nearest even) and inv_scale_dev
+ * is ignored.  inv_scale_dev holds 1 float (QCFG_PER_TENSOR) or `rows` floats (QCFG_PER_ROW).
+ * q_dev is [rows x ldq] elements (int8 or 2-byte bfloat16), 16-byte aligned, ldq a multiple
+ * of 16 and >= cols; columns cols..ldq-1 are zeroed.                                       */
+int qcfg_quantize(qcfg_ctx* ctx, const float* x_dev, int64_t rows, int64_t cols, int64_t ld,
+                  const float* inv_scale_dev, int granularity, int bits, void* q_dev,
+                  int64_t ldq, void* stream);
+
+/* Quantization-error sensitivity (Eq. 2) of n_tensors weight tensors for every bit width
+ * b_lo..b_hi (within 2..8) in ONE pass over the data.  w_dev, rows, cols are HOST arrays of
+ * length n_tensors (w_dev[t] a device pointer to a dense [rows[t] x cols[t]] fp32 matrix).
+ * Scales are max-calibrated per row (QCFG_PER_ROW) or per tensor.  Outputs, device memory:
+ * sse_dev[t*(b_hi-b_lo+1) + (b-b_lo)] = sum over the tensor of (x - Q_b(x))^2 (double) and
+ * absmax_dev[t] = max|x| over the tensor, so that
+ * E_QE(t, b) = sqrt(sse / (rows*cols)) / absmax.  Per-tensor granularity takes a second
+ * read of the tensor (the maximum must be known first).                                   */
+int qcfg_quant_error_sweep(qcfg_ctx* ctx, const float* const* w_dev, const int64_t* rows,
+                           const int64_t* cols, int32_t n_tensors, int granularity, int b_lo,
+                           int b_hi, double* sse_dev, float* absmax_dev, void* stream);
+
+/* One quantized GEMM with its fused epilogue, the kernel a configuration evaluation is made
+ * of: acc[m][n] = sum_k qx[m][k]*qw[n][k] (int8 x int8 -> int32, exact), then
+ * y = float(acc) * (scale_x * scale_w[n]) (the rescale of Eq. 1 for both operands), then
+ * the activation.  qx_dev is [m x ldx] int8, qw_dev [n x ldw] int8; ldx, ldw multiples of
+ * 16, pointers 16-byte aligned; columns k..ld-1 must be zero.  Either output may be NULL:
+ * y_dev [m x n] fp32, acc_dev [m x n] int32 (raw accumulators, for parity checks).         */
+int qcfg_gemm_i8(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t* qw_dev,
+                 int64_t ldw, int64_t m, int64_t n, int64_t k, float scale_x,
+                 const float* scale_w_dev, int act, float* y_dev, int32_t* acc_dev,
+                 void* stream);
+
+/* 16-bit layer (the paper's floating-point-16 baseline precision, Table 1):
+ * y = act(sum_k x[m][k]*w[n][k]) with bfloat16 operands (2-byte elements, leading
+ * dimensions multiples of 8 elements, padding zero) and fp32 accumulation.                */
+int qcfg_gemm_bf16(qcfg_ctx* ctx, const void* x_bf16_dev, int64_t ldx, const void* w_bf16_dev,
+                   int64_t ldw, int64_t m, int64_t n, int64_t k, int act, float* y_dev,
+                   void* stream);
+
+/* ---- model-level steps ---------------------------------------------------------------- */
+
+/* Builds a model from a HOST array of layers (copied).  Checks the graph: src and
+ * residual_from must point to earlier layers, k_in must fit the producer's slice.
+ * Weight maxima per output channel are computed here (one pass over every weight).        */
+int qcfg_model_create(qcfg_ctx* ctx, const qcfg_layer* layers, int32_t n_layers,
+                      qcfg_model** out);
+int qcfg_model_destroy(qcfg_model* model);
+
+/* Max calibration of every activation tensor (Section 3.1): a forward of x_dev ([m x k] fp32,
+ * or NHWC images with m = batch) with every layer at 16 bit -- the float model the searches
+ * start from -- recording max|input| of every layer.  Synchronises the stream and keeps the
+ * table on the host; QCFG_ENONFINITE if any maximum is NaN/Inf.                            */
+int qcfg_calibrate_model(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int64_t m,
+                         void* stream);
+/* Copies the calibrated activation maxima (n_layers floats) to a HOST array.              */
+int qcfg_model_act_absmax(qcfg_model* model, float* absmax_host);
+/* Copies layer `layer`'s per-row weight maxima (n_out floats) to a HOST array (syncs).    */
+int qcfg_model_weight_absmax(qcfg_model* model, int32_t layer, float* absmax_host);
+
+/* Evaluate f(x, w) (Algorithm 1 step "Evaluate f(x, lw)", Algorithm 2 "Evaluate f(x, w)"):
+ * forward of x_dev under the bit configuration bits[n_layers] (HOST array, values in
+ * {2..8, 16}).  Every layer quantizes its input with its calibrated activation scale at its
+ * own bit width (the clip of Eq. 1 is live), multiplies by its weight codes at that bit
+ * width (cached per (layer, b) after first use), rescales, adds the shortcut and applies the
+ * activation.  y_dev is a HOST array of n_layers DEVICE pointers; y_dev[l] receives layer l's
+ * fp32 output [rows_l x n_out] when non-NULL.  y_dev itself may be NULL (nothing returned;
+ * used when only throughput matters).                                                      */
+int qcfg_eval_config(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits,
+                     const float* x_dev, int64_t m, float* const* y_dev, void* stream);
+
+/* Parity taps for layer `layer` of the LAST qcfg_eval_config call (same stream order):
+ * the int8 codes of its GEMM input (qx_dev, [rows x k_in] dense, or NULL), of its weight
+ * (qw_dev, [n_out x k_in] dense, or NULL) and its raw int32 accumulators (acc_dev,
+ * [rows x n_out], or NULL; recomputed by a second GEMM launch).  QCFG_EBITS if that layer
+ * ran at 16 bit.                                                                           */
+int qcfg_debug_dump(qcfg_ctx* ctx, qcfg_model* model, int32_t layer, int8_t* qx_dev,
+                    int8_t* qw_dev, int32_t* acc_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QCFG_H_ */

@@ -1,0 +1,86 @@
+// Shared host/device helpers for the qcfg kernels (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/qcfg.h"
+
+namespace qcfg {
+
+// Device error word bits (ORed into the context's error word by kernels).
+enum : unsigned { ERR_TIMEOUT = 1u, ERR_NONFINITE = 2u };
+
+struct Ctx;  // defined in api.cu
+
+// ----- context services (api.cu) ------------------------------------------------------
+void count_launch(Ctx* ctx, int n = 1);
+int set_error(Ctx* ctx, int code, const char* fmt, ...);
+int check_cuda(Ctx* ctx, cudaError_t e, const char* what);
+unsigned* err_word(Ctx* ctx);
+int sm_count(Ctx* ctx);
+// grows (never shrinks) the context's scratch buffer; returns nullptr on failure
+void* scratch(Ctx* ctx, size_t bytes);
+
+// ----- elementwise.cu -----------------------------------------------------------------
+int launch_absmax(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t ld,
+                  int granularity, float* absmax, cudaStream_t st);
+int launch_scales(Ctx* ctx, const float* absmax, int64_t n, int bits, float* scale,
+                  float* inv_scale, cudaStream_t st);
+// inv_scale_ptr (device) or, when null, inv_scale_val for the whole tensor
+int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t ld,
+                    const float* inv_scale_ptr, float inv_scale_val, int granularity, int bits,
+                    void* q, int64_t ldq, cudaStream_t st);
+
+// ----- sweep.cu -----------------------------------------------------------------------
+int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
+                 int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse,
+                 float* absmax, cudaStream_t st);
+
+// ----- gemm.cu ------------------------------------------------------------------------
+constexpr int kMaxSlots = 3;
+struct CodeSlot {          // one fused re-quantize output of a GEMM epilogue
+  void* ptr;               // int8 (kind 1) or bf16 (kind 2) [m x ld]
+  int64_t ld;
+  float inv_scale;         // consumer's calibrated pre-rounding scale
+  float qmax;              // consumer's grid limit
+  int kind;                // 0 = unused
+};
+struct GemmArgs {
+  const void* a; int64_t lda;   // [m x lda] int8 or bf16, K-major
+  const void* b; int64_t ldb;   // [n x ldb]
+  int64_t m, n, k;
+  int is_bf16;
+  float scale_x;                // int8 only
+  const float* scale_w;         // int8 only, [n]
+  int act;
+  float* y; int64_t ldy;        // optional fp32 output
+  const float* residual; int64_t ldr;  // optional fp32 addend (before act)
+  int32_t* acc;                 // optional raw accumulators (int8 only) [m x n]
+  CodeSlot slots[kMaxSlots];
+};
+int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st);
+int gemm_init(Ctx* ctx);   // resolves the tensor-map encoder, sets smem attributes
+
+// ----- small device helpers -----------------------------------------------------------
+__device__ __forceinline__ unsigned warp_max_u(unsigned v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
+  }
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+// |x| as an unsigned integer: orders like the float for finite values, and NaN/Inf
+// compare above every finite value, so a max over these bits propagates them.
+__device__ __forceinline__ unsigned abs_bits(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+__host__ __device__ __forceinline__ float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
+
+}  // namespace qcfg
