@@ -1,0 +1,347 @@
+// Quantization-error sensitivity sweep (Eq. 2 of the paper): for every tensor and every bit
+// width b in 2..8 the sum of squared differences between x and Q_b(x), in ONE pass over HBM.
+//
+// A row (output channel) is held in registers by a team of 32..256 threads: the row maximum,
+// the 7 scale pairs and the 7 error sums all come from those registers, so every weight is
+// read from HBM exactly once.  Per element and bit width the work is four FMA-pipe ops:
+//   u = fma(x, inv_scale, 1.5*2^23)   (round-half-even of x*inv_scale in the low mantissa bits)
+//   r = u - 1.5*2^23                  (the code as a float)
+//   e = fma(-scale, r, x)             (x - Q(x))
+//   acc = fma(e, e, acc)
+// The clip of Eq. 1 is a no-op here because the scale comes from the row's own maximum.
+// Sums are fp32 within one row per thread, fp64 across rows, and reduced in a fixed order
+// (block partials in scratch memory, then one finalize block per tensor): deterministic.
+#include <vector>
+
+#include "common.cuh"
+
+namespace qcfg {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kNB = 7;                       // bit widths 2..8
+constexpr float kMagic = 12582912.0f;        // 1.5 * 2^23
+constexpr int kItemFloats = 32 * 1024;       // elements per work item (one block)
+
+struct SweepDesc {
+  const float* w;
+  int64_t rows;
+  int32_t cols;
+  int32_t item0;          // first work item (block) of this tensor within the launch
+  int32_t rows_per_item;
+  int32_t tensor;         // index into the caller's tensor list
+  int32_t team_log2;      // team size = 32 << team_log2
+  int32_t pad;
+};
+
+__device__ __forceinline__ const SweepDesc& find_desc(const SweepDesc* __restrict__ d, int n, int item) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (d[mid].item0 <= item) lo = mid; else hi = mid - 1;
+  }
+  return d[lo];
+}
+
+__device__ __forceinline__ void scales_for_lane(float A, int lane, float& s, float& inv) {
+  int b = 2 + (lane % kNB);
+  float qm = (float)((1 << (b - 1)) - 1);
+  s = 1.0f; inv = 1.0f;
+  if (A != 0.0f) { s = __fdiv_rn(A, qm); inv = __fdiv_rn(qm, A); }
+}
+
+__device__ __forceinline__ void err4(float x, float s, float inv, float& acc) {
+  float u = fmaf(x, inv, kMagic);
+  float r = u - kMagic;
+  float e = fmaf(-s, r, x);
+  acc = fmaf(e, e, acc);
+}
+
+// Writes the block's 7 sums and its maximum to partial[item*8 .. item*8+7].
+__device__ __forceinline__ void block_reduce_store(double (&dacc)[kNB], float amax, double* __restrict__ out) {
+  __shared__ double sred[kThreads / 32][8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int j = 0; j < kNB; ++j) {
+    double v = warp_sum(dacc[j]);
+    if (lane == 0) sred[warp][j] = v;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if (lane == 0) sred[warp][7] = (double)amax;
+  __syncthreads();
+  if (threadIdx.x < 8) {
+    double v = sred[0][threadIdx.x];
+    for (int w = 1; w < kThreads / 32; ++w)
+      v = (threadIdx.x == 7) ? fmax(v, sred[w][7]) : v + sred[w][threadIdx.x];
+    out[threadIdx.x] = v;
+  }
+}
+
+// Rows of up to 32*V*team float4; cols % 4 == 0 and 16-byte aligned rows.
+template <int V>
+__global__ void __launch_bounds__(kThreads, 2)
+sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tensor,
+                  const float* __restrict__ tensor_absmax, int jlo, int jhi,
+                  double* __restrict__ partial) {
+  const SweepDesc d = find_desc(descs, n_desc, blockIdx.x);
+  const int T = 32 << d.team_log2;
+  const int nteams = kThreads / T;
+  const int team = threadIdx.x / T;
+  const int tl = threadIdx.x % T;
+  const int lane = threadIdx.x & 31;
+  const int c4 = d.cols >> 2;
+  const int64_t row0 = (int64_t)(blockIdx.x - d.item0) * d.rows_per_item;
+  int64_t row1 = row0 + d.rows_per_item;
+  if (row1 > d.rows) row1 = d.rows;
+  const int n_iter = (int)((row1 - row0 + nteams - 1) / nteams);
+  const float A_tensor = per_tensor ? tensor_absmax[d.tensor] : 0.0f;
+
+  __shared__ float smax[kThreads / 32];
+
+  double dacc[kNB];
+#pragma unroll
+  for (int j = 0; j < kNB; ++j) dacc[j] = 0.0;
+  float amax_blk = 0.0f;
+
+  float4 cur[V], nxt[V];
+  auto load_row = [&](float4 (&dst)[V], int64_t row) {
+    const float4* p = reinterpret_cast<const float4*>(d.w + row * (int64_t)d.cols);
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      int c = tl + v * T;
+      dst[v] = (row < row1 && c < c4) ? __ldg(p + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  load_row(cur, row0 + team);
+
+  for (int it = 0; it < n_iter; ++it) {
+    load_row(nxt, row0 + (int64_t)(it + 1) * nteams + team);   // prefetch (zeros past the end)
+
+    float m = 0.0f;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+      m = fmaxf(fmaxf(fmaxf(m, fabsf(cur[v].x)), fmaxf(fabsf(cur[v].y), fabsf(cur[v].z))), fabsf(cur[v].w));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (T > 32) {
+      if (lane == 0) smax[threadIdx.x >> 5] = m;
+      __syncthreads();
+      const int w0 = team * (T >> 5);
+      m = smax[w0];
+      for (int w = 1; w < (T >> 5); ++w) m = fmaxf(m, smax[w0 + w]);
+      __syncthreads();
+    }
+    amax_blk = fmaxf(amax_blk, m);
+    if (per_tensor) m = A_tensor;
+
+    float s_l, inv_l;
+    scales_for_lane(m, lane, s_l, inv_l);
+    float s[kNB], inv[kNB], facc[kNB];
+#pragma unroll
+    for (int j = 0; j < kNB; ++j) {
+      s[j] = __shfl_sync(0xffffffffu, s_l, j);
+      inv[j] = __shfl_sync(0xffffffffu, inv_l, j);
+      facc[j] = 0.0f;
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+#pragma unroll
+      for (int j = 0; j < kNB; ++j) {
+        if (j >= jlo && j <= jhi) {
+          err4(cur[v].x, s[j], inv[j], facc[j]);
+          err4(cur[v].y, s[j], inv[j], facc[j]);
+          err4(cur[v].z, s[j], inv[j], facc[j]);
+          err4(cur[v].w, s[j], inv[j], facc[j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kNB; ++j) dacc[j] += (double)facc[j];
+#pragma unroll
+    for (int v = 0; v < V; ++v) cur[v] = nxt[v];
+  }
+  block_reduce_store(dacc, amax_blk, partial + (int64_t)blockIdx.x * 8);
+}
+
+// Any shape or alignment: the whole block works on one row at a time and reads it twice
+// (the second read hits L1/L2).
+__global__ void __launch_bounds__(kThreads)
+sweep_generic_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tensor,
+                     const float* __restrict__ tensor_absmax, int jlo, int jhi,
+                     double* __restrict__ partial) {
+  const SweepDesc d = find_desc(descs, n_desc, blockIdx.x);
+  const int lane = threadIdx.x & 31;
+  const int64_t row0 = (int64_t)(blockIdx.x - d.item0) * d.rows_per_item;
+  int64_t row1 = row0 + d.rows_per_item;
+  if (row1 > d.rows) row1 = d.rows;
+  const float A_tensor = per_tensor ? tensor_absmax[d.tensor] : 0.0f;
+  __shared__ float smax[kThreads / 32];
+  double dacc[kNB];
+#pragma unroll
+  for (int j = 0; j < kNB; ++j) dacc[j] = 0.0;
+  float amax_blk = 0.0f;
+  for (int64_t row = row0; row < row1; ++row) {
+    const float* p = d.w + row * (int64_t)d.cols;
+    float m = 0.0f;
+    for (int c = threadIdx.x; c < d.cols; c += kThreads) m = fmaxf(m, fabsf(__ldg(p + c)));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) smax[threadIdx.x >> 5] = m;
+    __syncthreads();
+    m = smax[0];
+    for (int w = 1; w < kThreads / 32; ++w) m = fmaxf(m, smax[w]);
+    __syncthreads();
+    amax_blk = fmaxf(amax_blk, m);
+    if (per_tensor) m = A_tensor;
+    float s_l, inv_l;
+    scales_for_lane(m, lane, s_l, inv_l);
+    float s[kNB], inv[kNB], facc[kNB];
+#pragma unroll
+    for (int j = 0; j < kNB; ++j) {
+      s[j] = __shfl_sync(0xffffffffu, s_l, j);
+      inv[j] = __shfl_sync(0xffffffffu, inv_l, j);
+      facc[j] = 0.0f;
+    }
+    for (int c = threadIdx.x; c < d.cols; c += kThreads) {
+      float x = __ldg(p + c);
+#pragma unroll
+      for (int j = 0; j < kNB; ++j)
+        if (j >= jlo && j <= jhi) err4(x, s[j], inv[j], facc[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < kNB; ++j) dacc[j] += (double)facc[j];
+  }
+  block_reduce_store(dacc, amax_blk, partial + (int64_t)blockIdx.x * 8);
+}
+
+struct TensorItems { int32_t item0, item1; };
+
+// One warp per tensor: sums the tensor's block partials in item order.
+__global__ void sweep_finalize_kernel(const double* __restrict__ partial, const TensorItems* __restrict__ ti,
+                                      int jlo, int nb, double* __restrict__ sse, float* __restrict__ absmax,
+                                      int write_absmax) {
+  const int t = blockIdx.x;
+  const int j = threadIdx.x;
+  const TensorItems r = ti[t];
+  if (j < nb) {
+    double v = 0.0;
+    for (int i = r.item0; i < r.item1; ++i) v += partial[(int64_t)i * 8 + jlo + j];
+    sse[(int64_t)t * nb + j] = v;
+  } else if (j == 31 && write_absmax) {
+    double v = 0.0;
+    for (int i = r.item0; i < r.item1; ++i) v = fmax(v, partial[(int64_t)i * 8 + 7]);
+    absmax[t] = (float)v;
+  }
+}
+
+template <int V>
+void launch_rows(const SweepDesc* d, int n, int items, int per_tensor, const float* amax, int jlo, int jhi,
+                 double* partial, cudaStream_t st) {
+  sweep_rows_kernel<V><<<items, kThreads, 0, st>>>(d, n, per_tensor, amax, jlo, jhi, partial);
+}
+
+}  // namespace
+
+int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols, int32_t n_tensors,
+                 int granularity, int b_lo, int b_hi, double* sse, float* absmax, cudaStream_t st) {
+  const int nb = b_hi - b_lo + 1;
+  const int per_tensor = granularity == QCFG_PER_TENSOR;
+  if (n_tensors == 0) return QCFG_OK;
+
+  // Group tensors by kernel variant: class 0 = generic, class V (1..8) = register-resident rows.
+  std::vector<SweepDesc> groups[9];
+  std::vector<TensorItems> titems(n_tensors);
+  for (int t = 0; t < n_tensors; ++t) {
+    SweepDesc d{};
+    d.w = w[t]; d.rows = rows[t]; d.cols = (int32_t)cols[t]; d.tensor = t;
+    int cls = 0;
+    const bool vec = ((uintptr_t)w[t] % 16 == 0) && (cols[t] % 4 == 0) && cols[t] <= 8192 && cols[t] > 0;
+    if (vec) {
+      int64_t c4 = cols[t] / 4;
+      int tl = 0;
+      while (tl < 3 && c4 > (int64_t)(32 << tl) * 8) ++tl;
+      d.team_log2 = tl;
+      cls = (int)((c4 + (32 << tl) - 1) / (32 << tl));     // float4 per thread, 1..8
+    }
+    int64_t rpi = cols[t] > 0 ? kItemFloats / cols[t] : 1;
+    if (cls > 0) {
+      int nteams = kThreads / (32 << d.team_log2);
+      rpi = (rpi / nteams) * nteams;
+      if (rpi < nteams) rpi = nteams;
+    }
+    if (rpi < 1) rpi = 1;
+    d.rows_per_item = (int32_t)rpi;
+    groups[cls].push_back(d);
+  }
+  // Assign work items: global numbering over all groups so every block owns one partial slot.
+  int total_items = 0;
+  int group_item0[9], group_items[9];
+  for (int c = 0; c < 9; ++c) {
+    group_item0[c] = total_items;
+    int local = 0;
+    for (auto& d : groups[c]) {
+      int n = (int)((d.rows + d.rows_per_item - 1) / d.rows_per_item);
+      d.item0 = local;
+      titems[d.tensor].item0 = total_items + local;
+      titems[d.tensor].item1 = total_items + local + n;
+      local += n;
+    }
+    group_items[c] = local;
+    total_items += local;
+  }
+
+  // Scratch layout: partials | descriptors (all groups) | tensor item ranges.
+  const size_t partial_bytes = (size_t)(total_items > 0 ? total_items : 1) * 8 * sizeof(double);
+  const size_t desc_bytes = (size_t)n_tensors * sizeof(SweepDesc);
+  const size_t ti_bytes = (size_t)n_tensors * sizeof(TensorItems);
+  char* base = static_cast<char*>(scratch(ctx, partial_bytes + desc_bytes + ti_bytes));
+  if (!base) return set_error(ctx, QCFG_ENOMEM, "sweep scratch (%zu bytes)", partial_bytes + desc_bytes + ti_bytes);
+  double* partial = reinterpret_cast<double*>(base);
+  SweepDesc* ddev = reinterpret_cast<SweepDesc*>(base + partial_bytes);
+  TensorItems* tidev = reinterpret_cast<TensorItems*>(base + partial_bytes + desc_bytes);
+
+  std::vector<SweepDesc> flat;
+  int group_desc0[9];
+  for (int c = 0; c < 9; ++c) {
+    group_desc0[c] = (int)flat.size();
+    flat.insert(flat.end(), groups[c].begin(), groups[c].end());
+  }
+  cudaError_t e = cudaMemcpyAsync(ddev, flat.data(), desc_bytes, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(tidev, titems.data(), ti_bytes, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "sweep descriptor upload");
+
+  if (per_tensor) {
+    for (int t = 0; t < n_tensors; ++t) {
+      int rc = launch_absmax(ctx, w[t], rows[t], cols[t], cols[t], QCFG_PER_TENSOR, absmax + t, st);
+      if (rc != QCFG_OK) return rc;
+    }
+  }
+  const int jlo = b_lo - 2, jhi = b_hi - 2;
+  for (int c = 0; c < 9; ++c) {
+    if (group_items[c] == 0) continue;
+    const SweepDesc* d = ddev + group_desc0[c];
+    const int n = (int)groups[c].size();
+    double* part = partial + (int64_t)group_item0[c] * 8;
+    switch (c) {
+      case 0: sweep_generic_kernel<<<group_items[c], kThreads, 0, st>>>(d, n, per_tensor, absmax, jlo, jhi, part); break;
+      case 1: launch_rows<1>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 2: launch_rows<2>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 3: launch_rows<3>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 4: launch_rows<4>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 5: launch_rows<5>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 6: launch_rows<6>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 7: launch_rows<7>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      default: launch_rows<8>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+    }
+    count_launch(ctx);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return check_cuda(ctx, e, "sweep launch");
+  }
+  sweep_finalize_kernel<<<n_tensors, 32, 0, st>>>(partial, tidev, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "sweep finalize launch");
+}
+
+}  // namespace qcfg
