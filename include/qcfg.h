@@ -82,6 +82,11 @@ const char* qcfg_last_error(qcfg_ctx* ctx);
 /* Number of kernels this context has launched since creation (for accounting).            */
 int64_t qcfg_launch_count(qcfg_ctx* ctx);
 
+/* Switches the fusion of the consumer's quantize step into the producing GEMM's epilogue
+ * (default on).  Off: every layer's fp32 output is written and re-read by a separate quantize
+ * kernel; results are bit-identical either way.                                           */
+int qcfg_set_fusion(qcfg_ctx* ctx, int enabled);
+
 /* ---- tensor-level steps --------------------------------------------------------------- */
 
 /* Max calibration (Section 3.1: the maximum value of each tensor; absolute value as in

@@ -1,0 +1,571 @@
+// C-ABI of the library: context, model (layer table, weight-code cache, calibration tables)
+// and the host planner that turns one bit configuration into a sequence of kernel launches.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace qcfg {
+
+struct Ctx {
+  int device = 0;
+  int sms = 0;
+  unsigned* err_dev = nullptr;
+  void* scratch_buf = nullptr;
+  size_t scratch_bytes = 0;
+  int64_t launches = 0;
+  int fuse = 1;
+  char msg[512] = {0};
+};
+
+void count_launch(Ctx* ctx, int n) { ctx->launches += n; }
+unsigned* err_word(Ctx* ctx) { return ctx->err_dev; }
+int sm_count(Ctx* ctx) { return ctx->sms; }
+
+int set_error(Ctx* ctx, int code, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->msg, sizeof(ctx->msg), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+int check_cuda(Ctx* ctx, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return QCFG_OK;
+  return set_error(ctx, e == cudaErrorMemoryAllocation ? QCFG_ENOMEM : QCFG_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+void* scratch(Ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->scratch_bytes) return ctx->scratch_buf;
+  // the old buffer may still be in use by queued work on some stream
+  if (ctx->scratch_buf) { cudaDeviceSynchronize(); cudaFree(ctx->scratch_buf); ctx->scratch_buf = nullptr; ctx->scratch_bytes = 0; }
+  size_t want = bytes + bytes / 4 + 4096;
+  void* p = nullptr;
+  if (cudaMalloc(&p, want) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  ctx->scratch_buf = p;
+  ctx->scratch_bytes = want;
+  return p;
+}
+
+namespace {
+
+inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline bool bits_int(int b) { return b >= 2 && b <= 8; }
+inline bool bits_ok(int b) { return bits_int(b) || b == 16; }
+
+struct DevBuf {
+  void* p = nullptr;
+  size_t bytes = 0;
+  int ensure(Ctx* ctx, size_t want) {
+    if (want <= bytes) return QCFG_OK;
+    if (p) { cudaDeviceSynchronize(); cudaFree(p); p = nullptr; bytes = 0; }
+    cudaError_t e = cudaMalloc(&p, want);
+    if (e != cudaSuccess) { cudaGetLastError(); p = nullptr; return set_error(ctx, QCFG_ENOMEM, "cudaMalloc of %zu bytes failed", want); }
+    bytes = want;
+    return QCFG_OK;
+  }
+  void release() { if (p) cudaFree(p); p = nullptr; bytes = 0; }
+};
+
+struct WeightCodes {
+  DevBuf codes;           // int8 or bf16 [n_out x ldk]
+  DevBuf scale;           // fp32 [n_out] post-rounding scales (int only)
+  DevBuf inv;             // fp32 [n_out] pre-rounding scales (int only)
+  bool ready = false;
+};
+
+struct LayerState {
+  qcfg_layer d;
+  int64_t ldk = 0;                 // padded k_in of the code matrices
+  DevBuf w_absmax;                 // fp32 [n_out]
+  WeightCodes wc[17];              // by bit width
+  float act_absmax = 0.0f;         // calibrated max|input|
+  std::vector<int> consumers;      // layers reading this layer's output as GEMM input
+  bool feeds_residual = false;
+  // per-evaluation state
+  int64_t rows = 0;
+  DevBuf ybuf;                     // internal fp32 output [rows x n_out]
+  DevBuf abuf;                     // GEMM input codes [rows x ldk] (sized for bf16)
+  DevBuf prebuf;                   // pooled fp32 input (convolution table only)
+  const void* a_ptr = nullptr;     // codes actually used (may alias another layer's abuf)
+  const float* y_ptr = nullptr;    // where this layer's fp32 output went (nullptr: not materialised)
+  bool a_ready = false;
+  int bits = 0;
+};
+
+}  // namespace
+
+struct Model {
+  Ctx* ctx = nullptr;
+  std::vector<LayerState> L;
+  bool calibrated = false;
+  bool evaluated = false;
+  DevBuf act_absmax_dev;           // fp32 [n_layers], filled by calibration
+  int64_t last_m = 0;
+};
+
+namespace {
+
+int64_t layer_rows(const Model* M, int l, int64_t m_ext) {
+  const qcfg_layer& d = M->L[l].d;
+  if (d.kh > 0) {
+    int64_t oh = (d.in_h + 2 * d.pad - d.kh) / d.stride + 1;
+    int64_t ow = (d.in_w + 2 * d.pad - d.kw) / d.stride + 1;
+    return m_ext * oh * ow;
+  }
+  if (d.pool_before == QCFG_POOL_GLOBAL_AVG) return m_ext;
+  return d.src < 0 ? m_ext : layer_rows(M, d.src, m_ext);
+}
+
+bool is_plain_linear(const qcfg_layer& d) { return d.kh == 0 && d.pool_before == QCFG_POOL_NONE; }
+
+// Weight codes and per-row scales for (layer, bits); computed once and kept.
+int ensure_weight_codes(Ctx* ctx, LayerState& S, int bits, cudaStream_t st) {
+  WeightCodes& W = S.wc[bits];
+  if (W.ready) return QCFG_OK;
+  const int64_t n = S.d.n_out, k = S.d.k_in;
+  int rc = W.codes.ensure(ctx, (size_t)(n * S.ldk) * (bits == 16 ? 2 : 1));
+  if (rc) return rc;
+  if (bits == 16) {
+    rc = launch_quantize(ctx, S.d.w_dev, n, k, k, nullptr, 1.0f, QCFG_PER_ROW, 16, W.codes.p, S.ldk, st);
+  } else {
+    rc = W.scale.ensure(ctx, (size_t)n * 4);
+    if (!rc) rc = W.inv.ensure(ctx, (size_t)n * 4);
+    if (!rc) rc = launch_scales(ctx, (const float*)S.w_absmax.p, n, bits, (float*)W.scale.p, (float*)W.inv.p, st);
+    if (!rc) rc = launch_quantize(ctx, S.d.w_dev, n, k, k, (const float*)W.inv.p, 1.0f, QCFG_PER_ROW, bits, W.codes.p, S.ldk, st);
+  }
+  if (rc) return rc;
+  W.ready = true;
+  return QCFG_OK;
+}
+
+// Host copy of the scale rule (one IEEE fp32 division each; the device kernels use __fdiv_rn).
+inline void host_scales(float A, int bits, float* scale, float* inv) {
+  const float qm = qmax_of(bits);
+  if (A == 0.0f) { *scale = 1.0f; *inv = 1.0f; return; }
+  volatile float s = A / qm, i = qm / A;
+  *scale = s; *inv = i;
+}
+
+struct Source { const float* p; int64_t ld; };
+
+// Row length of the external input: widest slice any layer reads from it (channels for images).
+int64_t ext_ld_of(const Model* M) {
+  int64_t ld = 0;
+  for (auto& S : M->L) {
+    if (S.d.src >= 0) continue;
+    int64_t w = S.d.kh > 0 ? S.d.in_c : S.d.src_col0 + S.d.k_in;
+    if (w > ld) ld = w;
+  }
+  return ld;
+}
+
+// fp32 matrix a plain-linear layer reads (slice of its producer's output or of the input).
+int linear_source(Model* M, int l, const float* x_dev, Source* out) {
+  LayerState& S = M->L[l];
+  if (S.d.src < 0) { out->p = x_dev + S.d.src_col0; out->ld = S.d.k_in + 0; return QCFG_OK; }
+  LayerState& P = M->L[S.d.src];
+  if (!P.y_ptr) return set_error(M->ctx, QCFG_ESTATE, "layer %d: producer %d output not materialised", l, S.d.src);
+  out->p = P.y_ptr + S.d.src_col0;
+  out->ld = P.d.n_out;
+  return QCFG_OK;
+}
+
+// One forward pass.  calibrate = true: every layer at 16 bit, record max|input| per layer.
+int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t x_ld, int64_t m,
+            float* const* y_dev, bool calibrate, cudaStream_t st) {
+  const int n = (int)M->L.size();
+  for (int l = 0; l < n; ++l) {
+    LayerState& S = M->L[l];
+    S.rows = layer_rows(M, l, m);
+    S.a_ready = false; S.a_ptr = nullptr; S.y_ptr = nullptr;
+    S.bits = calibrate ? 16 : bits[l];
+    if (!is_plain_linear(S.d) || S.d.residual_from >= 0)
+      return set_error(ctx, QCFG_EUNIMPL, "layer %d: convolution / pooling / shortcut layers are not available in this build", l);
+  }
+  for (int l = 0; l < n; ++l) {
+    LayerState& S = M->L[l];
+    const int b = S.bits;
+    int rc = ensure_weight_codes(ctx, S, b, st);
+    if (rc) return rc;
+
+    // ---- GEMM input codes
+    if (!S.a_ready) {
+      Source src;
+      if (S.d.src < 0) { src.p = x_dev + S.d.src_col0; src.ld = x_ld; }
+      else if ((rc = linear_source(M, l, x_dev, &src))) return rc;
+      if (calibrate) {
+        rc = launch_absmax(ctx, src.p, S.rows, S.d.k_in, src.ld, QCFG_PER_TENSOR, (float*)M->act_absmax_dev.p + l, st);
+        if (rc) return rc;
+      }
+      // reuse the codes of an earlier layer that reads the same slice with the same grid
+      int share = -1;
+      for (int j = 0; j < l && share < 0; ++j) {
+        LayerState& T = M->L[j];
+        if (T.d.src == S.d.src && T.d.src_col0 == S.d.src_col0 && T.d.k_in == S.d.k_in && T.bits == b &&
+            T.a_ptr && (b == 16 || T.act_absmax == S.act_absmax))
+          share = j;
+      }
+      if (share >= 0) {
+        S.a_ptr = M->L[share].a_ptr;
+      } else {
+        rc = S.abuf.ensure(ctx, (size_t)(S.rows * S.ldk) * 2);
+        if (rc) return rc;
+        float sc = 1.0f, inv = 1.0f;
+        if (b != 16) host_scales(S.act_absmax, b, &sc, &inv);
+        rc = launch_quantize(ctx, src.p, S.rows, S.d.k_in, src.ld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
+        if (rc) return rc;
+        S.a_ptr = S.abuf.p;
+      }
+      S.a_ready = true;
+    }
+
+    // ---- GEMM + epilogue
+    GemmArgs g{};
+    g.a = S.a_ptr; g.lda = S.ldk;
+    g.b = S.wc[b].codes.p; g.ldb = S.ldk;
+    g.m = S.rows; g.n = S.d.n_out; g.k = S.d.k_in;
+    g.is_bf16 = b == 16;
+    g.act = S.d.act;
+    if (b != 16) {
+      float sx, ix;
+      host_scales(S.act_absmax, b, &sx, &ix);
+      g.scale_x = sx;
+      g.scale_w = (const float*)S.wc[b].scale.p;
+    }
+    // fused re-quantize outputs for consumers whose input is this whole output
+    bool all_fused = !S.consumers.empty();
+    int nslots = 0;
+    for (int c : S.consumers) {
+      LayerState& C = M->L[c];
+      const int cb = calibrate ? 16 : bits[c];
+      const bool fusable = ctx->fuse && !calibrate && is_plain_linear(C.d) && C.d.src_col0 == 0 && C.d.k_in == S.d.n_out;
+      if (!fusable) { all_fused = false; continue; }
+      float csc = 1.0f, cinv = 1.0f;
+      if (cb != 16) host_scales(C.act_absmax, cb, &csc, &cinv);
+      // an existing slot with the same grid serves this consumer too
+      int found = -1;
+      for (int s = 0; s < nslots; ++s)
+        if ((cb == 16 && g.slots[s].kind == 2) || (cb != 16 && g.slots[s].kind == 1 && g.slots[s].inv_scale == cinv && g.slots[s].qmax == qmax_of(cb)))
+          found = s;
+      if (found < 0) {
+        if (nslots == kMaxSlots) { all_fused = false; continue; }
+        rc = C.abuf.ensure(ctx, (size_t)(S.rows * C.ldk) * 2);
+        if (rc) return rc;
+        g.slots[nslots].ptr = C.abuf.p;
+        g.slots[nslots].ld = C.ldk;
+        g.slots[nslots].inv_scale = cinv;
+        g.slots[nslots].qmax = cb == 16 ? 0.0f : qmax_of(cb);
+        g.slots[nslots].kind = cb == 16 ? 2 : 1;
+        found = nslots++;
+      }
+      C.a_ptr = g.slots[found].ptr;
+      C.a_ready = true;
+      C.bits = cb;
+    }
+    float* y_out = (y_dev && y_dev[l]) ? y_dev[l] : nullptr;
+    const bool need_y = y_out || !all_fused || S.feeds_residual;
+    if (need_y && !y_out) {
+      rc = S.ybuf.ensure(ctx, (size_t)(S.rows * S.d.n_out) * 4);
+      if (rc) return rc;
+      y_out = (float*)S.ybuf.p;
+    }
+    g.y = y_out; g.ldy = S.d.n_out;
+    S.y_ptr = y_out;
+    rc = launch_gemm(ctx, g, st);
+    if (rc) return rc;
+  }
+  return QCFG_OK;
+}
+
+}  // namespace
+}  // namespace qcfg
+
+using namespace qcfg;
+
+struct qcfg_ctx { Ctx c; };
+struct qcfg_model { Model m; };
+
+extern "C" {
+
+int qcfg_create(qcfg_ctx** out, int device) {
+  if (!out) return QCFG_EINVAL;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) { cudaGetLastError(); return QCFG_ECUDA; }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return QCFG_ECUDA;
+  if (prop.major != 10) return QCFG_EARCH;
+  if (cudaSetDevice(device) != cudaSuccess) return QCFG_ECUDA;
+  qcfg_ctx* h = new (std::nothrow) qcfg_ctx();
+  if (!h) return QCFG_ENOMEM;
+  h->c.device = device;
+  h->c.sms = prop.multiProcessorCount;
+  if (cudaMalloc(&h->c.err_dev, sizeof(unsigned)) != cudaSuccess || cudaMemset(h->c.err_dev, 0, sizeof(unsigned)) != cudaSuccess) {
+    delete h;
+    return QCFG_ENOMEM;
+  }
+  int rc = gemm_init(&h->c);
+  if (rc) { cudaFree(h->c.err_dev); delete h; return rc; }
+  *out = h;
+  return QCFG_OK;
+}
+
+int qcfg_destroy(qcfg_ctx* ctx) {
+  if (!ctx) return QCFG_EINVAL;
+  cudaDeviceSynchronize();
+  if (ctx->c.scratch_buf) cudaFree(ctx->c.scratch_buf);
+  if (ctx->c.err_dev) cudaFree(ctx->c.err_dev);
+  delete ctx;
+  return QCFG_OK;
+}
+
+int qcfg_sync_status(qcfg_ctx* ctx, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return check_cuda(c, e, "stream synchronize");
+  unsigned w = 0;
+  e = cudaMemcpy(&w, c->err_dev, sizeof(w), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return check_cuda(c, e, "error word read");
+  if (w) {
+    cudaMemset(c->err_dev, 0, sizeof(w));
+    if (w & ERR_TIMEOUT) return set_error(c, QCFG_ETIMEOUT, "a bounded device-side wait gave up");
+    if (w & ERR_NONFINITE) return set_error(c, QCFG_ENONFINITE, "non-finite value found on the device");
+  }
+  return QCFG_OK;
+}
+
+const char* qcfg_last_error(qcfg_ctx* ctx) { return ctx ? ctx->c.msg : "null context"; }
+int64_t qcfg_launch_count(qcfg_ctx* ctx) { return ctx ? ctx->c.launches : 0; }
+int qcfg_set_fusion(qcfg_ctx* ctx, int enabled) {
+  if (!ctx) return QCFG_EINVAL;
+  ctx->c.fuse = enabled ? 1 : 0;
+  return QCFG_OK;
+}
+
+int qcfg_calibrate(qcfg_ctx* ctx, const float* x_dev, int64_t rows, int64_t cols, int64_t ld, int granularity,
+                   float* absmax_dev, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!absmax_dev || rows < 0 || cols < 0 || (rows * cols > 0 && !x_dev)) return set_error(c, QCFG_EINVAL, "calibrate: null pointer or negative size");
+  if (granularity != QCFG_PER_TENSOR && granularity != QCFG_PER_ROW) return set_error(c, QCFG_EINVAL, "calibrate: bad granularity");
+  if (ld < cols) return set_error(c, QCFG_ESHAPE, "calibrate: ld < cols");
+  if ((uintptr_t)x_dev % 4 || (uintptr_t)absmax_dev % 4) return set_error(c, QCFG_EALIGN, "calibrate: pointers must be 4-byte aligned");
+  return launch_absmax(c, x_dev, rows, cols, ld, granularity, absmax_dev, (cudaStream_t)stream);
+}
+
+int qcfg_scales_from_absmax(qcfg_ctx* ctx, const float* absmax_dev, int64_t n, int bits, float* scale_dev,
+                            float* inv_scale_dev, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!absmax_dev || n < 0) return set_error(c, QCFG_EINVAL, "scales: null pointer or negative size");
+  if (!bits_int(bits)) return set_error(c, QCFG_EBITS, "scales: bits must be 2..8, got %d", bits);
+  return launch_scales(c, absmax_dev, n, bits, scale_dev, inv_scale_dev, (cudaStream_t)stream);
+}
+
+int qcfg_quantize(qcfg_ctx* ctx, const float* x_dev, int64_t rows, int64_t cols, int64_t ld, const float* inv_scale_dev,
+                  int granularity, int bits, void* q_dev, int64_t ldq, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!x_dev || !q_dev || rows < 0 || cols < 0) return set_error(c, QCFG_EINVAL, "quantize: null pointer or negative size");
+  if (!bits_ok(bits)) return set_error(c, QCFG_EBITS, "quantize: bits must be 2..8 or 16, got %d", bits);
+  if (bits != 16 && !inv_scale_dev) return set_error(c, QCFG_EINVAL, "quantize: inv_scale_dev is null");
+  if (granularity != QCFG_PER_TENSOR && granularity != QCFG_PER_ROW) return set_error(c, QCFG_EINVAL, "quantize: bad granularity");
+  if (ld < cols || ldq < cols) return set_error(c, QCFG_ESHAPE, "quantize: leading dimension below cols");
+  if (ldq % 16 || (uintptr_t)q_dev % 16 || (uintptr_t)x_dev % 4) return set_error(c, QCFG_EALIGN, "quantize: q_dev must be 16-byte aligned with ldq a multiple of 16");
+  return launch_quantize(c, x_dev, rows, cols, ld, inv_scale_dev, 1.0f, granularity, bits, q_dev, ldq, (cudaStream_t)stream);
+}
+
+int qcfg_quant_error_sweep(qcfg_ctx* ctx, const float* const* w_dev, const int64_t* rows, const int64_t* cols,
+                           int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse_dev, float* absmax_dev,
+                           void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (n_tensors < 0 || !sse_dev || !absmax_dev || (n_tensors > 0 && (!w_dev || !rows || !cols)))
+    return set_error(c, QCFG_EINVAL, "sweep: null pointer or negative count");
+  if (!bits_int(b_lo) || !bits_int(b_hi) || b_lo > b_hi) return set_error(c, QCFG_EBITS, "sweep: bit range must lie in 2..8");
+  if (granularity != QCFG_PER_TENSOR && granularity != QCFG_PER_ROW) return set_error(c, QCFG_EINVAL, "sweep: bad granularity");
+  for (int t = 0; t < n_tensors; ++t) {
+    if (rows[t] < 0 || cols[t] < 0 || cols[t] > 0x7fffffff) return set_error(c, QCFG_ESHAPE, "sweep: tensor %d has a bad shape", t);
+    if (rows[t] * cols[t] > 0 && !w_dev[t]) return set_error(c, QCFG_EINVAL, "sweep: tensor %d is null", t);
+    if ((uintptr_t)w_dev[t] % 4) return set_error(c, QCFG_EALIGN, "sweep: tensor %d is not 4-byte aligned", t);
+  }
+  return launch_sweep(c, w_dev, rows, cols, n_tensors, granularity, b_lo, b_hi, sse_dev, absmax_dev, (cudaStream_t)stream);
+}
+
+int qcfg_gemm_i8(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t* qw_dev, int64_t ldw, int64_t m,
+                 int64_t n, int64_t k, float scale_x, const float* scale_w_dev, int act, float* y_dev, int32_t* acc_dev,
+                 void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!qx_dev || !qw_dev || (!y_dev && !acc_dev) || (y_dev && !scale_w_dev)) return set_error(c, QCFG_EINVAL, "gemm_i8: null pointer");
+  if (act < QCFG_ACT_NONE || act > QCFG_ACT_GELU_TANH) return set_error(c, QCFG_EINVAL, "gemm_i8: bad activation");
+  if ((uintptr_t)y_dev % 4 || (uintptr_t)acc_dev % 4 || (uintptr_t)scale_w_dev % 4) return set_error(c, QCFG_EALIGN, "gemm_i8: outputs must be 4-byte aligned");
+  GemmArgs g{};
+  g.a = qx_dev; g.lda = ldx; g.b = qw_dev; g.ldb = ldw; g.m = m; g.n = n; g.k = k;
+  g.is_bf16 = 0; g.scale_x = scale_x; g.scale_w = scale_w_dev; g.act = act;
+  g.y = y_dev; g.ldy = n; g.acc = acc_dev;
+  if (!scale_w_dev) {   // accumulators only: the rescale is skipped by giving it nothing to write
+    g.y = nullptr;
+  }
+  return launch_gemm(c, g, (cudaStream_t)stream);
+}
+
+int qcfg_gemm_bf16(qcfg_ctx* ctx, const void* x_bf16_dev, int64_t ldx, const void* w_bf16_dev, int64_t ldw, int64_t m,
+                   int64_t n, int64_t k, int act, float* y_dev, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!x_bf16_dev || !w_bf16_dev || !y_dev) return set_error(c, QCFG_EINVAL, "gemm_bf16: null pointer");
+  if (act < QCFG_ACT_NONE || act > QCFG_ACT_GELU_TANH) return set_error(c, QCFG_EINVAL, "gemm_bf16: bad activation");
+  if ((uintptr_t)y_dev % 4) return set_error(c, QCFG_EALIGN, "gemm_bf16: y_dev must be 4-byte aligned");
+  GemmArgs g{};
+  g.a = x_bf16_dev; g.lda = ldx; g.b = w_bf16_dev; g.ldb = ldw; g.m = m; g.n = n; g.k = k;
+  g.is_bf16 = 1; g.act = act; g.y = y_dev; g.ldy = n;
+  return launch_gemm(c, g, (cudaStream_t)stream);
+}
+
+int qcfg_model_create(qcfg_ctx* ctx, const qcfg_layer* layers, int32_t n_layers, qcfg_model** out) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!out) return set_error(c, QCFG_EINVAL, "model_create: out is null");
+  *out = nullptr;
+  if (!layers || n_layers <= 0) return set_error(c, QCFG_EINVAL, "model_create: no layers");
+  for (int l = 0; l < n_layers; ++l) {
+    const qcfg_layer& d = layers[l];
+    if (!d.w_dev || d.n_out <= 0 || d.k_in <= 0) return set_error(c, QCFG_EINVAL, "layer %d: null weight or empty shape", l);
+    if ((uintptr_t)d.w_dev % 4) return set_error(c, QCFG_EALIGN, "layer %d: weight pointer not 4-byte aligned", l);
+    if (d.src >= l || d.src < -1 || d.residual_from >= l || d.residual_from < -1) return set_error(c, QCFG_ESHAPE, "layer %d: src / residual_from must be earlier layers", l);
+    if (d.act < QCFG_ACT_NONE || d.act > QCFG_ACT_GELU_TANH) return set_error(c, QCFG_EINVAL, "layer %d: bad activation", l);
+    if (d.src_col0 < 0) return set_error(c, QCFG_ESHAPE, "layer %d: negative src_col0", l);
+    if (d.kh == 0 && d.pool_before == QCFG_POOL_NONE && d.src >= 0 && d.src_col0 + d.k_in > layers[d.src].n_out)
+      return set_error(c, QCFG_ESHAPE, "layer %d: reads columns beyond its producer's output", l);
+    if (d.kh > 0 && (d.kw <= 0 || d.stride <= 0 || d.pad < 0 || d.in_h <= 0 || d.in_w <= 0 || d.in_c <= 0 ||
+                     (int64_t)d.kh * d.kw * d.in_c != d.k_in))
+      return set_error(c, QCFG_ESHAPE, "layer %d: inconsistent convolution geometry", l);
+    if (d.residual_from >= 0 && layers[d.residual_from].n_out != d.n_out) return set_error(c, QCFG_ESHAPE, "layer %d: shortcut width differs", l);
+  }
+  qcfg_model* h = new (std::nothrow) qcfg_model();
+  if (!h) return set_error(c, QCFG_ENOMEM, "model_create: host allocation failed");
+  Model* M = &h->m;
+  M->ctx = c;
+  M->L.resize(n_layers);
+  int rc = M->act_absmax_dev.ensure(c, (size_t)n_layers * 4);
+  for (int l = 0; l < n_layers && !rc; ++l) {
+    LayerState& S = M->L[l];
+    S.d = layers[l];
+    S.ldk = round_up(S.d.k_in, 16);
+    if (S.d.src >= 0) M->L[S.d.src].consumers.push_back(l);
+    if (S.d.residual_from >= 0) M->L[S.d.residual_from].feeds_residual = true;
+    rc = S.w_absmax.ensure(c, (size_t)S.d.n_out * 4);
+    if (!rc) rc = launch_absmax(c, S.d.w_dev, S.d.n_out, S.d.k_in, S.d.k_in, QCFG_PER_ROW, (float*)S.w_absmax.p, 0);
+  }
+  if (!rc) rc = check_cuda(c, cudaStreamSynchronize(0), "model_create sync");
+  if (rc) { qcfg_model_destroy(h); return rc; }
+  *out = h;
+  return QCFG_OK;
+}
+
+int qcfg_model_destroy(qcfg_model* model) {
+  if (!model) return QCFG_EINVAL;
+  cudaDeviceSynchronize();
+  Model* M = &model->m;
+  for (auto& S : M->L) {
+    S.w_absmax.release(); S.ybuf.release(); S.abuf.release(); S.prebuf.release();
+    for (auto& W : S.wc) { W.codes.release(); W.scale.release(); W.inv.release(); }
+  }
+  M->act_absmax_dev.release();
+  delete model;
+  return QCFG_OK;
+}
+
+int qcfg_calibrate_model(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int64_t m, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  if (!x_dev || m <= 0) return set_error(c, QCFG_EINVAL, "calibrate_model: null input or m <= 0");
+  if ((uintptr_t)x_dev % 4) return set_error(c, QCFG_EALIGN, "calibrate_model: x_dev not 4-byte aligned");
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t ext_ld = ext_ld_of(M);
+  int rc = forward(c, M, nullptr, x_dev, ext_ld, m, nullptr, true, st);
+  if (rc) return rc;
+  std::vector<float> host(M->L.size());
+  rc = check_cuda(c, cudaMemcpyAsync(host.data(), M->act_absmax_dev.p, host.size() * 4, cudaMemcpyDeviceToHost, st), "calibration table copy");
+  if (!rc) rc = qcfg_sync_status(ctx, stream);
+  if (rc) return rc;
+  for (size_t l = 0; l < host.size(); ++l)
+    if (!std::isfinite(host[l])) return set_error(c, QCFG_ENONFINITE, "layer %zu: calibrated input maximum is not finite", l);
+  for (size_t l = 0; l < host.size(); ++l) M->L[l].act_absmax = host[l];
+  M->calibrated = true;
+  M->evaluated = false;
+  return QCFG_OK;
+}
+
+int qcfg_model_act_absmax(qcfg_model* model, float* absmax_host) {
+  if (!model || !absmax_host) return QCFG_EINVAL;
+  if (!model->m.calibrated) return QCFG_ESTATE;
+  for (size_t l = 0; l < model->m.L.size(); ++l) absmax_host[l] = model->m.L[l].act_absmax;
+  return QCFG_OK;
+}
+
+int qcfg_model_weight_absmax(qcfg_model* model, int32_t layer, float* absmax_host) {
+  if (!model || !absmax_host) return QCFG_EINVAL;
+  Model* M = &model->m;
+  if (layer < 0 || layer >= (int)M->L.size()) return set_error(M->ctx, QCFG_EINVAL, "weight_absmax: bad layer index");
+  LayerState& S = M->L[layer];
+  return check_cuda(M->ctx, cudaMemcpy(absmax_host, S.w_absmax.p, (size_t)S.d.n_out * 4, cudaMemcpyDeviceToHost), "weight maxima copy");
+}
+
+int qcfg_eval_config(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, const float* x_dev, int64_t m,
+                     float* const* y_dev, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  if (!bits || !x_dev || m <= 0) return set_error(c, QCFG_EINVAL, "eval_config: null pointer or m <= 0");
+  if (!M->calibrated) return set_error(c, QCFG_ESTATE, "eval_config: model is not calibrated");
+  if ((uintptr_t)x_dev % 4) return set_error(c, QCFG_EALIGN, "eval_config: x_dev not 4-byte aligned");
+  for (size_t l = 0; l < M->L.size(); ++l) {
+    if (!bits_ok(bits[l])) return set_error(c, QCFG_EBITS, "eval_config: layer %zu has bit width %d", l, (int)bits[l]);
+    if (y_dev && y_dev[l] && (uintptr_t)y_dev[l] % 4) return set_error(c, QCFG_EALIGN, "eval_config: y_dev[%zu] not 4-byte aligned", l);
+  }
+  const int64_t ext_ld = ext_ld_of(M);
+  int rc = forward(c, M, bits, x_dev, ext_ld, m, y_dev, false, (cudaStream_t)stream);
+  if (rc) return rc;
+  M->evaluated = true;
+  M->last_m = m;
+  return QCFG_OK;
+}
+
+int qcfg_debug_dump(qcfg_ctx* ctx, qcfg_model* model, int32_t layer, int8_t* qx_dev, int8_t* qw_dev, int32_t* acc_dev,
+                    void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  if (!M->evaluated) return set_error(c, QCFG_ESTATE, "debug_dump: no evaluation has run");
+  if (layer < 0 || layer >= (int)M->L.size()) return set_error(c, QCFG_EINVAL, "debug_dump: bad layer index");
+  LayerState& S = M->L[layer];
+  if (!bits_int(S.bits)) return set_error(c, QCFG_EBITS, "debug_dump: layer %d ran at %d bit", layer, S.bits);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (qx_dev) {
+    cudaError_t e = cudaMemcpy2DAsync(qx_dev, (size_t)S.d.k_in, S.a_ptr, (size_t)S.ldk, (size_t)S.d.k_in, (size_t)S.rows, cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return check_cuda(c, e, "debug_dump qx copy");
+  }
+  if (qw_dev) {
+    cudaError_t e = cudaMemcpy2DAsync(qw_dev, (size_t)S.d.k_in, S.wc[S.bits].codes.p, (size_t)S.ldk, (size_t)S.d.k_in, (size_t)S.d.n_out, cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return check_cuda(c, e, "debug_dump qw copy");
+  }
+  if (acc_dev) {
+    GemmArgs g{};
+    g.a = S.a_ptr; g.lda = S.ldk; g.b = S.wc[S.bits].codes.p; g.ldb = S.ldk;
+    g.m = S.rows; g.n = S.d.n_out; g.k = S.d.k_in; g.acc = acc_dev;
+    g.scale_x = 1.0f; g.scale_w = (const float*)S.wc[S.bits].scale.p;
+    return launch_gemm(c, g, st);
+  }
+  return QCFG_OK;
+}
+
+}  // extern "C"

@@ -43,6 +43,7 @@ struct GemmParams {
   float* y; int64_t ldy;
   const float* residual; int64_t ldr;
   int32_t* acc;
+  int32_t need_y;             // anything besides raw accumulators to produce
   CodeSlot slots[kMaxSlots];
   unsigned* err;
 };
@@ -187,6 +188,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, uint32_t (&v
     }
   }
 
+  if (!p.need_y) return;
   float y[32];
   if (BF16) {
 #pragma unroll
@@ -466,7 +468,10 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   p.idesc = ((g.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
   p.scale_x = g.scale_x; p.scale_w = g.scale_w; p.act = g.act;
   p.y = g.y; p.ldy = g.ldy; p.residual = g.residual; p.ldr = g.ldr; p.acc = g.acc;
-  for (int s = 0; s < kMaxSlots; ++s) p.slots[s] = g.slots[s];
+  p.need_y = g.y != nullptr;
+  for (int s = 0; s < kMaxSlots; ++s) { p.slots[s] = g.slots[s]; if (g.slots[s].kind) p.need_y = 1; }
+  if (!p.need_y && !g.acc) return set_error(ctx, QCFG_EINVAL, "gemm: no output requested");
+  if (p.need_y && !g.is_bf16 && !g.scale_w) return set_error(ctx, QCFG_EINVAL, "gemm: scale_w is null");
   p.err = err_word(ctx);
 
   CUtensorMap ma, mb;

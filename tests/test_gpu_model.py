@@ -1,0 +1,176 @@
+"""Parity of whole configuration evaluations with the CPU oracle, through the C-ABI.
+
+Primary gate: layer-wise teacher forcing.  For every layer the test downloads the fp32
+input the GPU actually fed to it, lets the oracle recompute scale, codes, int32 accumulators
+and output from that input, and requires codes, scale bit patterns and accumulators to be
+bit-exact, outputs to be bit-exact (no activation / ReLU), within 1e-6 relative with a floor
+of 1e-6 * max|y| (GELU), or within 1e-2 normwise (16-bit layers).  End-to-end chained outputs
+are compared with float tolerances; the ReLU-only integer model must be bit-exact end to end.
+"""
+import numpy as np
+import pytest
+import torch
+
+import qcfg_workloads as wl
+from oracle import qcfg_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2302_01382_b200 as q
+    c = q.Context(0)
+    yield c
+    c.close()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def host(t):
+    return t.detach().cpu().numpy()
+
+
+def build(ctx, w):
+    import paper_2302_01382_b200 as q
+    weights = [dev(a) for a in w.weights]
+    model = q.Model(ctx, w.layers, weights)
+    x = dev(w.x.reshape(w.x.shape[0], -1) if w.x.ndim == 2 else w.x)
+    model.calibrate_model(x, w.m)
+    return model, x
+
+
+def run_eval(ctx, model, w, x, bits):
+    ys = [torch.full((wl.layer_rows(w.layers, l, w.m), lay.n_out), float("nan"), device="cuda")
+          for l, lay in enumerate(w.layers)]
+    model.eval_config(bits, x, w.m, ys)
+    ctx.check_sync()
+    return ys
+
+
+def check_calibration(model, w):
+    act_o, w_o = orc.calibrate_model(w.layers, w.weights, w.x)
+    act_g = np.array(model.act_absmax(), np.float32)
+    # the 16-bit forward accumulates in fp32 on the GPU and fp64 in the oracle: maxima agree to
+    # bf16-product accumulation accuracy, not bit for bit (except for external inputs)
+    for l, lay in enumerate(w.layers):
+        if lay.src < 0 and lay.pool_before == 0:
+            assert act_g[l] == act_o[l]
+        else:
+            assert act_g[l] == pytest.approx(float(act_o[l]), rel=2e-3)
+        np.testing.assert_array_equal(np.array(model.weight_absmax(l), np.float32), w_o[l])
+    return act_g, w_o
+
+
+def teacher_forced_check(ctx, model, w, x, bits, ys, act_g, w_amax, sample_rows=None):
+    outs = [host(y) for y in ys]
+    for o in outs:
+        assert np.all(np.isfinite(o)), "an output element was never written"
+    for l, lay in enumerate(w.layers):
+        b = int(bits[l])
+        xin = orc.layer_input(w.layers, l, w.x, outs)          # built from the GPU's own outputs
+        res = outs[lay.residual_from] if lay.residual_from >= 0 else None
+        rows = None
+        if sample_rows is not None and outs[l].shape[0] > sample_rows:
+            rows = np.sort(np.random.default_rng(l).choice(outs[l].shape[0], sample_rows, replace=False))
+        y_ref, taps = orc.eval_layer_teacher_forced(lay, w.weights[l], xin, b, act_g[l], w_amax[l], residual=res, rows=rows)
+        y_gpu = outs[l] if rows is None else outs[l][rows]
+        if b == 16:
+            assert np.linalg.norm(y_gpu - y_ref) <= 1e-2 * max(np.linalg.norm(y_ref), 1e-30), l
+            assert np.abs(y_gpu - y_ref).max() <= 1e-2 * max(np.abs(y_ref).max(), 1e-30), l
+            continue
+        m_rows, k = outs[l].shape[0], lay.k_in
+        qx = torch.empty((m_rows, k), dtype=torch.int8, device="cuda")
+        qw = torch.empty((lay.n_out, k), dtype=torch.int8, device="cuda")
+        acc = torch.empty((m_rows, lay.n_out), dtype=torch.int32, device="cuda")
+        model.debug_dump(l, qx, qw, acc)
+        ctx.check_sync()
+        qx, acc = host(qx), host(acc)
+        if rows is not None:
+            qx, acc = qx[rows], acc[rows]
+        np.testing.assert_array_equal(qx, taps["qx"], err_msg=f"layer {l} input codes")
+        np.testing.assert_array_equal(host(qw), taps["qw"], err_msg=f"layer {l} weight codes")
+        np.testing.assert_array_equal(acc, taps["acc"], err_msg=f"layer {l} accumulators")
+        if lay.act == orc.ACT_GELU_TANH:
+            np.testing.assert_allclose(y_gpu, y_ref, rtol=1e-6, atol=1e-6 * np.abs(y_ref).max(), err_msg=f"layer {l}")
+        else:
+            np.testing.assert_array_equal(y_gpu.view(np.uint32), y_ref.view(np.uint32), err_msg=f"layer {l}")
+
+
+def test_tiny_mlp_bit_exact_end_to_end(ctx):
+    w = wl.tiny_mlp()
+    model, x = build(ctx, w)
+    act_g, w_amax = check_calibration(model, w)
+    ys = run_eval(ctx, model, w, x, w.bits)
+    teacher_forced_check(ctx, model, w, x, w.bits, ys, act_g, w_amax)
+    # chained oracle with the GPU's calibration table: integers and ReLU only -> bit-exact
+    outs = orc.eval_config(w.layers, w.weights, w.bits, w.x, list(act_g), w_amax)
+    for l in range(3):
+        np.testing.assert_array_equal(host(ys[l]), outs[l])
+    model.close()
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+@pytest.mark.parametrize("seed,m,hidden,ffn,blocks", [(11, 300, 192, 768, 2), (12, 1100, 256, 1024, 1)])
+def test_bert_stack_teacher_forced(ctx, fuse, seed, m, hidden, ffn, blocks):
+    ctx.set_fusion(fuse)
+    try:
+        w = wl.bert_stack(seed, m, hidden, ffn, blocks)
+        model, x = build(ctx, w)
+        act_g, w_amax = check_calibration(model, w)
+        for bits in (w.bits, [8] * len(w.layers), [4, 8, 16, 3, 16, 2] * blocks):
+            ys = run_eval(ctx, model, w, x, bits)
+            teacher_forced_check(ctx, model, w, x, bits, ys, act_g, w_amax)
+            # end to end against the chained oracle: float tolerance only (GELU, bf16 layers)
+            outs = orc.eval_config(w.layers, w.weights, bits, w.x, list(act_g), w_amax)
+            last = host(ys[-1])
+            assert np.linalg.norm(last - outs[-1]) <= 2e-2 * np.linalg.norm(outs[-1])
+        model.close()
+    finally:
+        ctx.set_fusion(True)
+
+
+def test_fused_and_unfused_agree_bitwise_and_taps_are_optional(ctx):
+    w = wl.bert_stack(21, 515, 128, 512, 2, bit_choices=(4, 8))
+    model, x = build(ctx, w)
+    ys_f = run_eval(ctx, model, w, x, w.bits)
+    ctx.set_fusion(False)
+    ys_u = run_eval(ctx, model, w, x, w.bits)
+    ctx.set_fusion(True)
+    for a, b in zip(ys_f, ys_u):
+        assert torch.equal(a, b)
+    # only the last layer requested: same values
+    ys = [None] * (len(w.layers) - 1) + [torch.empty_like(ys_f[-1])]
+    model.eval_config(w.bits, x, w.m, ys)
+    ctx.check_sync()
+    assert torch.equal(ys[-1], ys_f[-1])
+    model.eval_config(w.bits, x, w.m, None)
+    ctx.check_sync()
+    model.close()
+
+
+def test_model_argument_errors(ctx):
+    import paper_2302_01382_b200 as q
+    w = wl.tiny_mlp()
+    weights = [dev(a) for a in w.weights]
+    model = q.Model(ctx, w.layers, weights)
+    x = dev(w.x)
+    with pytest.raises(q.QcfgError) as e:
+        model.eval_config(w.bits, x, w.m)
+    assert e.value.status == q.ESTATE
+    model.calibrate_model(x, w.m)
+    with pytest.raises(q.QcfgError) as e:
+        model.eval_config([8, 9, 8], x, w.m)
+    assert e.value.status == q.EBITS
+    bad = [wl.Layer("a", 8, 16), wl.Layer("b", 8, 16, src=0)]      # reads 16 columns of an 8-wide output
+    with pytest.raises(q.QcfgError) as e:
+        q.Model(ctx, bad, [torch.zeros((8, 16), device="cuda")] * 2)
+    assert e.value.status == q.ESHAPE
+    xn = x.clone()
+    xn[3, 3] = float("nan")
+    with pytest.raises(q.QcfgError) as e:
+        model.calibrate_model(xn, w.m)
+    assert e.value.status == q.ENONFINITE
+    model.close()
