@@ -235,7 +235,7 @@ def test_argument_errors_leave_outputs_untouched(ctx):
         ctx.quantize(x, x[0], q.PER_TENSOR, 12)
     assert e.value.status == q.EBITS
     with pytest.raises(q.QcfgError) as e:
-        ctx.quantize(x, x[0], q.PER_TENSOR, 8, ldq=24)
+        ctx.quantize(x, x[0], q.PER_TENSOR, 8, ldq=40)
     assert e.value.status == q.EALIGN
     with pytest.raises(q.QcfgError) as e:
         ctx.quant_error_sweep([x], b_lo=1, b_hi=8)
