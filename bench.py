@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the bit-configuration evaluator on one B200 (or N independent replicas).
+
+Workload (the third configuration of the benchmark list): a 12-block BERT-base-shaped stack
+of 72 linear tensors.  One STEP is one whole job of the hot path over one batch of synthetic
+input: the quantization-error sweep (b = 2..8, per output channel) over all 72 weights, max
+calibration of the model on the batch (a 16-bit forward), then the 72 configuration
+evaluations of one greedy pass at 32 x 384 tokens, each lowering one tensor from 8 to 4 bits
+in the order the sweep gives, with a scripted accept/reject stream.  The metric is
+configuration evaluations per second over the whole job.
+
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line (rank 0).
+`--impl reference` times the CPU oracle instead (a bounded sample per step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import qcfg_workloads as wl  # noqa: E402
+
+METRIC = "config_evals_per_sec"
+UNIT = "evals/s"
+N_EVALS = 72
+TOKENS = 32 * 384
+WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value: float, world: int) -> float:
+    """Max of a per-rank scalar over all ranks (torch.distributed must be initialised if world > 1)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([value], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [s.strip() for s in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample(w, rows: int, n_sweep_tensors: int):
+    """A bounded sample of one job on the CPU oracle: the sweep over the first tensors, plus
+    calibration and ONE configuration evaluation on the first `rows` tokens.  Returns
+    (seconds of the evaluation part, seconds of the sweep part, elements swept)."""
+    from oracle import qcfg_oracle as orc
+    t0 = time.perf_counter()
+    orc.quant_error_sweep(w.weights[:n_sweep_tensors], orc.PER_ROW)
+    t_sweep = time.perf_counter() - t0
+    elems = sum(a.size for a in w.weights[:n_sweep_tensors])
+    x = w.x[:rows]
+    act, wmax = orc.calibrate_model(w.layers, w.weights, x)
+    bits = np.full(len(w.layers), 8, np.uint8)
+    bits[::7] = 4
+    t0 = time.perf_counter()
+    orc.eval_config(w.layers, w.weights, bits, x, act, wmax)
+    t_eval = time.perf_counter() - t0
+    return t_eval, t_sweep, elems
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    rows, n_sweep = 768, 6
+    w = wl.bert_base_x12()
+    for _ in range(max(args.warmup, 0) and 1):
+        oracle_sample(w, 128, 1)
+    t_evals, t_sweeps = [], []
+    t_all0 = time.perf_counter()
+    for _ in range(args.steps):
+        te, ts, elems = oracle_sample(w, rows, n_sweep)
+        t_evals.append(te); t_sweeps.append(ts)
+    wall = time.perf_counter() - t_all0
+    te = float(np.mean(t_evals))
+    evals_per_s = (rows / TOKENS) / te            # one full-size evaluation takes te * TOKENS / rows
+    cores = cpu_threads()
+    sample = (f"per step: one evaluation of the 72-layer stack on the first {rows} of {TOKENS} tokens "
+              f"(scaled by rows) and the sweep over the first {n_sweep} of 72 tensors")
+    line = {"impl": "reference", "metric": METRIC, "value": evals_per_s, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(args.steps, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8/f64",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "tokens": TOKENS, "evals_per_step": N_EVALS},
+            "cpu_baseline": {"value": evals_per_s, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "sweep_gbs": 4e-9 * elems / float(np.mean(t_sweeps))},
+            "e2e": {"value": evals_per_s, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ GPU arm
+
+class Job:
+    """Device-resident state of the benchmark job and the code of one step."""
+
+    def __init__(self, q, ctx, w, torch):
+        self.q, self.ctx, self.w, self.torch = q, ctx, w, torch
+        self.weights = [torch.from_numpy(a).cuda() for a in w.weights]
+        self.x = torch.from_numpy(w.x).cuda()
+        self.model = q.Model(ctx, w.layers, self.weights)
+        self.sse = torch.empty((len(self.weights), 7), dtype=torch.float64, device="cuda")
+        self.amax = torch.empty(len(self.weights), dtype=torch.float32, device="cuda")
+        self.sizes = np.array([a.size for a in w.weights], dtype=np.float64)
+        self.out = torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32, device="cuda")
+        self.ys = [None] * (len(w.layers) - 1) + [self.out]
+        self.last_ranking = None
+
+    def ranking_from_sweep(self):
+        sse = self.sse.cpu().numpy()           # synchronises: the search order needs the sweep result
+        amax = self.amax.cpu().numpy().astype(np.float64)
+        eqe = np.sqrt(sse[:, 2] / self.sizes) / np.where(amax > 0, amax, 1.0)   # E_QE at b = 4
+        return np.argsort(eqe, kind="stable")
+
+    def step(self, x=None, host_out=None):
+        ctx, w = self.ctx, self.w
+        x = self.x if x is None else x
+        ctx.quant_error_sweep(self.weights, self.q.PER_ROW, 2, 8, sse=self.sse, absmax=self.amax)
+        rank = self.ranking_from_sweep()
+        self.last_ranking = rank
+        self.model.calibrate_model(x, w.m)
+        for bits in wl.greedy_sequence(rank, w.accept):
+            self.model.eval_config(bits, x, w.m, self.ys)
+            if host_out is not None:
+                host_out.copy_(self.out, non_blocking=True)
+
+
+def run_gpu(args):
+    import torch
+    import paper_2302_01382_b200 as q
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        torch.cuda.set_device(0)
+    dev_index = torch.cuda.current_device()
+    ctx = q.Context(dev_index)
+    peaks = load_peaks()
+
+    w = wl.bert_base_x12()
+    job = Job(q, ctx, w, torch)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- device-resident timing (value)
+    for _ in range(args.warmup):
+        job.step()
+    ctx.check_sync()
+    ctx.profile_enable(True)
+    ctx.profile_read(0); ctx.profile_read(1)
+    launches0 = ctx.launch_count()
+    sampler = ClockSampler(dev_index)
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        job.step()
+    e1.record()
+    barrier()
+    ctx.check_sync()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world)
+    clocks = sampler.stop()
+    launches = ctx.launch_count() - launches0
+    g_ms, g_n, g_ops = ctx.profile_read(0)
+    b_ms, b_n, b_ops = ctx.profile_read(1)
+    ctx.profile_enable(False)
+    value = world * N_EVALS * args.steps / (ms_total * 1e-3)
+
+    # ---------------- sweep alone (sub-metric), L2 flushed by its own 340 MB input
+    sw0, sw1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_sw = 10
+    sw0.record()
+    for _ in range(n_sw):
+        ctx.quant_error_sweep(job.weights, q.PER_ROW, 2, 8, sse=job.sse, absmax=job.amax)
+    sw1.record()
+    torch.cuda.synchronize()
+    sweep_ms = sw0.elapsed_time(sw1) / n_sw
+    sweep_bytes = 4.0 * float(job.sizes.sum())
+    sweep_gbs = sweep_bytes / (sweep_ms * 1e-3) / 1e9
+
+    # ---------------- end to end: host buffers, copies inside the timed region
+    host_x = torch.from_numpy(w.x).pin_memory()
+    host_out = torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32).pin_memory()
+    x_dev = torch.empty_like(job.x)
+    e2e_steps = max(1, min(args.steps, 3))
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(e2e_steps):
+        x_dev.copy_(host_x, non_blocking=True)
+        job.step(x_dev, host_out)
+    t1.record()
+    barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1), world)
+    e2e_value = world * N_EVALS * e2e_steps / (e2e_ms * 1e-3)
+    h2d = host_x.numel() * 4
+    d2h = N_EVALS * host_out.numel() * 4 + job.sse.numel() * 8 + job.amax.numel() * 4 + 4 * len(w.layers)
+
+    if rank == 0:
+        int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])
+        achieved = (g_ops / max(g_n, 1)) / (g_ms / max(g_n, 1) * 1e-3) / 1e12 if g_n else 0.0
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens": TOKENS, "evals_per_step": N_EVALS, "layers": len(w.layers),
+                       "l2": "inputs larger than L2 (340 MB weights, 38 MB activations per layer)",
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "steps": e2e_steps},
+            "roofline": {"kernel": "gemm_kernel<int8>", "bound": "tensor", "achieved": achieved, "peak": int8_peak,
+                         "unit": "TOP/s", "frac": achieved / int8_peak,
+                         "peak_source": f"2 x sustained bf16 cuBLAS ({peaks['_source']})",
+                         "launches": int(g_n), "avg_launch_us": 1e3 * g_ms / max(g_n, 1), "traffic": None},
+            "sweep": {"gbs": sweep_gbs, "ms": sweep_ms, "bytes": sweep_bytes, "hbm_peak_gbs": peaks["hbm_gbs"],
+                      "frac": sweep_gbs / peaks["hbm_gbs"], "peak_source": peaks["_source"]},
+            "gemm_bf16": {"tflops": (b_ops / (b_ms * 1e-3) / 1e12) if b_ms else None, "launches": int(b_n)},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            te, ts, elems = oracle_sample(w, 768, 6)
+            line["cpu_baseline"] = {"value": (768 / TOKENS) / te, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                    "sample": "one evaluation of the 72-layer stack on the first 768 of 12288 tokens "
+                                              "(scaled by rows); sweep over the first 6 of 72 tensors",
+                                    "sweep_gbs": 4e-9 * elems / ts}
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -87,6 +87,15 @@ int64_t qcfg_launch_count(qcfg_ctx* ctx);
  * kernel; results are bit-identical either way.                                           */
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled);
 
+/* Per-launch timing of the GEMM kernel with CUDA events recorded on the launching stream
+ * (off by default; a few microseconds of host time per launch when on).  kernel_class 0 is
+ * the int8 GEMM, 1 the bf16 GEMM.  qcfg_profile_read waits for the recorded launches, then
+ * returns the summed kernel time (ms), the number of launches and the summed algorithmic
+ * operations (2*m*n*k per launch) since the last reset.  Outputs may be NULL.            */
+int qcfg_profile_enable(qcfg_ctx* ctx, int enabled);
+int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* launches, double* ops,
+                      int reset);
+
 /* ---- tensor-level steps --------------------------------------------------------------- */
 
 /* Max calibration (Section 3.1: the maximum value of each tensor; absolute value as in

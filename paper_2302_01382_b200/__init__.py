@@ -22,7 +22,7 @@ STATUS_NAMES = ["OK", "EINVAL", "EBITS", "ESHAPE", "EALIGN", "ENOMEM", "ENONFINI
 EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT, EUNIMPL, ESTATE = range(1, 12)
 
 EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error", "qcfg_launch_count",
-           "qcfg_set_fusion", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
+           "qcfg_set_fusion", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_gemm_i8", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
            "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_debug_dump"]
@@ -60,6 +60,8 @@ def load_library() -> C.CDLL:
         "qcfg_destroy": [vp],
         "qcfg_sync_status": [vp, vp],
         "qcfg_set_fusion": [vp, ci],
+        "qcfg_profile_enable": [vp, ci],
+        "qcfg_profile_read": [vp, ci, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double), ci],
         "qcfg_calibrate": [vp, vp, i64, i64, i64, ci, vp, vp],
         "qcfg_scales_from_absmax": [vp, vp, i64, ci, vp, vp, vp],
         "qcfg_quantize": [vp, vp, i64, i64, i64, vp, ci, ci, vp, i64, vp],
@@ -137,6 +139,14 @@ class Context:
 
     def set_fusion(self, enabled: bool):
         self._check(self.lib.qcfg_set_fusion(self.h, int(enabled)))
+
+    def profile_enable(self, enabled: bool):
+        self._check(self.lib.qcfg_profile_enable(self.h, int(enabled)))
+
+    def profile_read(self, kernel_class: int, reset: bool = True):
+        ms, n, ops = C.c_double(), C.c_int64(), C.c_double()
+        self._check(self.lib.qcfg_profile_read(self.h, kernel_class, C.byref(ms), C.byref(n), C.byref(ops), int(reset)))
+        return ms.value, n.value, ops.value
 
     # ---- tensor-level steps
     def calibrate(self, x: torch.Tensor, granularity: int, out: Optional[torch.Tensor] = None, stream=None):

@@ -20,7 +20,41 @@ struct Ctx {
   int64_t launches = 0;
   int fuse = 1;
   char msg[512] = {0};
+  // per-launch event timing (off by default)
+  int prof = 0;
+  std::vector<cudaEvent_t> ev;      // pairs: ev[2i] before, ev[2i+1] after
+  std::vector<int> ev_cls;
+  size_t ev_used = 0;               // pairs in flight
+  double prof_ms[2] = {0, 0}, prof_ops[2] = {0, 0};
+  int64_t prof_n[2] = {0, 0};
 };
+
+constexpr size_t kProfPairs = 8192;
+
+static void prof_drain(Ctx* ctx) {
+  if (ctx->ev_used == 0) return;
+  cudaEventSynchronize(ctx->ev[2 * ctx->ev_used - 1]);
+  for (size_t i = 0; i < ctx->ev_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->ev[2 * i], ctx->ev[2 * i + 1]) == cudaSuccess) {
+      ctx->prof_ms[ctx->ev_cls[i]] += ms;
+      ctx->prof_n[ctx->ev_cls[i]] += 1;
+    }
+  }
+  ctx->ev_used = 0;
+}
+void prof_begin(Ctx* ctx, int cls, cudaStream_t st) {
+  if (!ctx->prof) return;
+  if (ctx->ev_used == kProfPairs) prof_drain(ctx);
+  ctx->ev_cls[ctx->ev_used] = cls;
+  cudaEventRecord(ctx->ev[2 * ctx->ev_used], st);
+}
+void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st) {
+  if (!ctx->prof) return;
+  cudaEventRecord(ctx->ev[2 * ctx->ev_used + 1], st);
+  ctx->prof_ops[cls] += ops;
+  ctx->ev_used += 1;
+}
 
 void count_launch(Ctx* ctx, int n) { ctx->launches += n; }
 unsigned* err_word(Ctx* ctx) { return ctx->err_dev; }
@@ -318,6 +352,7 @@ int qcfg_create(qcfg_ctx** out, int device) {
 int qcfg_destroy(qcfg_ctx* ctx) {
   if (!ctx) return QCFG_EINVAL;
   cudaDeviceSynchronize();
+  for (auto& e : ctx->c.ev) cudaEventDestroy(e);
   if (ctx->c.scratch_buf) cudaFree(ctx->c.scratch_buf);
   if (ctx->c.err_dev) cudaFree(ctx->c.err_dev);
   delete ctx;
@@ -342,6 +377,29 @@ int qcfg_sync_status(qcfg_ctx* ctx, void* stream) {
 
 const char* qcfg_last_error(qcfg_ctx* ctx) { return ctx ? ctx->c.msg : "null context"; }
 int64_t qcfg_launch_count(qcfg_ctx* ctx) { return ctx ? ctx->c.launches : 0; }
+int qcfg_profile_enable(qcfg_ctx* ctx, int enabled) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (enabled && c->ev.empty()) {
+    c->ev.resize(2 * kProfPairs);
+    c->ev_cls.resize(kProfPairs);
+    for (auto& e : c->ev)
+      if (cudaEventCreate(&e) != cudaSuccess) return set_error(c, QCFG_ECUDA, "profile: event creation failed");
+  }
+  if (!enabled) prof_drain(c);
+  c->prof = enabled ? 1 : 0;
+  return QCFG_OK;
+}
+int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* launches, double* ops, int reset) {
+  if (!ctx || kernel_class < 0 || kernel_class > 1) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  prof_drain(c);
+  if (ms) *ms = c->prof_ms[kernel_class];
+  if (launches) *launches = c->prof_n[kernel_class];
+  if (ops) *ops = c->prof_ops[kernel_class];
+  if (reset) { c->prof_ms[kernel_class] = 0; c->prof_n[kernel_class] = 0; c->prof_ops[kernel_class] = 0; }
+  return QCFG_OK;
+}
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled) {
   if (!ctx) return QCFG_EINVAL;
   ctx->c.fuse = enabled ? 1 : 0;

@@ -22,6 +22,9 @@ unsigned* err_word(Ctx* ctx);
 int sm_count(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);
+// optional per-launch timing of one kernel class (0 = int8 GEMM, 1 = bf16 GEMM) with CUDA events
+void prof_begin(Ctx* ctx, int cls, cudaStream_t st);
+void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st);
 
 // ----- elementwise.cu -----------------------------------------------------------------
 int launch_absmax(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t ld,

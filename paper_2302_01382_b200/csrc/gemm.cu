@@ -483,8 +483,10 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   int grid = sm_count(ctx);
   if (grid > num_tiles) grid = num_tiles;
   const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)stages * stage_bytes;
+  prof_begin(ctx, g.is_bf16 ? 1 : 0, st);
   if (g.is_bf16) gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(ma, mb, p);
   else gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(ma, mb, p);
+  prof_end(ctx, g.is_bf16 ? 1 : 0, 2.0 * (double)g.m * (double)g.n * (double)g.k, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "gemm launch");
 }
