@@ -133,6 +133,31 @@ int qcfg_quant_error_sweep(qcfg_ctx* ctx, const float* const* w_dev, const int64
                            const int64_t* cols, int32_t n_tensors, int granularity, int b_lo,
                            int b_hi, double* sse_dev, float* absmax_dev, void* stream);
 
+/* The same sweep for callers that cannot allocate device memory when they call: code that
+ * runs after a serving engine or training framework has reserved all of the GPU's memory for
+ * its own pool (so cudaMalloc would fail), or inside a latency-critical loop where the implicit
+ * device-wide synchronisation of cudaMalloc/cudaFree is not acceptable.  (The paper has no
+ * counterpart; this is a deployment variant of qcfg_quant_error_sweep.)  Arguments, outputs and
+ * results are those of qcfg_quant_error_sweep.  Differences:
+ *   - Its scratch memory (block partial sums and descriptor tables) is a fixed array inside
+ *     the library image, about 1.05 MiB on every GPU that loads the library, held until the
+ *     process exits.  The call itself performs no cudaMalloc, cudaFree or other device allocation.
+ *   - Limits per call: at most 1024 tensors and at most 16384 work items, one work item being
+ *     up to 32768 elements of one tensor (rows are not split), i.e. roughly 512 Mi elements.
+ *     Anything larger returns QCFG_ENOMEM with a message and does nothing; split the tensors
+ *     over several calls, one after the other.
+ *   - ctx's device must be the current device (QCFG_ESTATE otherwise).  The first call on a
+ *     device looks up the array's device address (cudaGetSymbolAddress) and keeps it; make
+ *     that first call during start-up, before any stream capture begins.
+ *   - All calls, from every context and stream of the process, share that one array per GPU.
+ *     A call overwrites what the previous call left (nothing needs clearing: every value read is
+ *     written first by the same call), so two calls must not overlap on the GPU: issue them on
+ *     one stream, or order them with events.  Overlapping calls race and give wrong sums.     */
+int qcfg_quant_error_sweep_static(qcfg_ctx* ctx, const float* const* w_dev, const int64_t* rows,
+                                  const int64_t* cols, int32_t n_tensors, int granularity,
+                                  int b_lo, int b_hi, double* sse_dev, float* absmax_dev,
+                                  void* stream);
+
 /* One quantized GEMM with its fused epilogue, the kernel a configuration evaluation is made
  * of: acc[m][n] = sum_k qx[m][k]*qw[n][k] (int8 x int8 -> int32, exact), then
  * y = float(acc) * (scale_x * scale_w[n]) (the rescale of Eq. 1 for both operands), then

@@ -23,7 +23,7 @@ EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT, EUNIM
 
 EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error", "qcfg_launch_count",
            "qcfg_set_fusion", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
-           "qcfg_quant_error_sweep", "qcfg_gemm_i8", "qcfg_gemm_bf16", "qcfg_model_create",
+           "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
            "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_debug_dump"]
 
@@ -66,6 +66,7 @@ def load_library() -> C.CDLL:
         "qcfg_scales_from_absmax": [vp, vp, i64, ci, vp, vp, vp],
         "qcfg_quantize": [vp, vp, i64, i64, i64, vp, ci, ci, vp, i64, vp],
         "qcfg_quant_error_sweep": [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), i32, ci, ci, ci, vp, vp, vp],
+        "qcfg_quant_error_sweep_static": [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), i32, ci, ci, ci, vp, vp, vp],
         "qcfg_gemm_i8": [vp, vp, i64, vp, i64, i64, i64, i64, f32, vp, ci, vp, vp, vp],
         "qcfg_gemm_bf16": [vp, vp, i64, vp, i64, i64, i64, i64, ci, vp, vp],
         "qcfg_model_create": [vp, C.POINTER(LayerStruct), i32, C.POINTER(vp)],
@@ -186,6 +187,28 @@ class Context:
         cols = (C.c_int64 * max(n, 1))(*[t.shape[1] for t in tensors])
         self._check(self.lib.qcfg_quant_error_sweep(self.h, ptrs, rows, cols, n, granularity, b_lo, b_hi, _ptr(sse),
                                                     _ptr(absmax), _stream(stream)))
+        return sse, absmax
+
+    def quant_error_sweep_static(self, tensors: Sequence[torch.Tensor], granularity: int = PER_ROW, b_lo: int = 2,
+                                 b_hi: int = 8, sse: Optional[torch.Tensor] = None, absmax: Optional[torch.Tensor] = None,
+                                 shapes: Optional[Sequence] = None, stream=None):
+        """The sweep through the entry point that allocates no device memory (fixed scratch array
+        inside the library, shared by all calls: do not overlap two of them on the GPU).  Pass
+        `sse` and `absmax` to keep the binding from allocating either.  `shapes` overrides the
+        (rows, cols) taken from the tensors."""
+        n = len(tensors)
+        nb = b_hi - b_lo + 1
+        dev = tensors[0].device if n else torch.device("cuda", self.device)
+        if sse is None:
+            sse = torch.empty((n, nb), dtype=torch.float64, device=dev)
+        if absmax is None:
+            absmax = torch.empty(n, dtype=torch.float32, device=dev)
+        shp = shapes if shapes is not None else [tuple(t.shape) for t in tensors]
+        ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in tensors])
+        rows = (C.c_int64 * max(n, 1))(*[s[0] for s in shp])
+        cols = (C.c_int64 * max(n, 1))(*[s[1] for s in shp])
+        self._check(self.lib.qcfg_quant_error_sweep_static(self.h, ptrs, rows, cols, n, granularity, b_lo, b_hi,
+                                                           _ptr(sse), _ptr(absmax), _stream(stream)))
         return sse, absmax
 
     def gemm_i8(self, qx: torch.Tensor, qw: torch.Tensor, k: int, scale_x: float, scale_w: Optional[torch.Tensor],

@@ -59,6 +59,7 @@ void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st) {
 void count_launch(Ctx* ctx, int n) { ctx->launches += n; }
 unsigned* err_word(Ctx* ctx) { return ctx->err_dev; }
 int sm_count(Ctx* ctx) { return ctx->sms; }
+int device_of(Ctx* ctx) { return ctx->device; }
 
 int set_error(Ctx* ctx, int code, const char* fmt, ...) {
   if (ctx) {
@@ -454,6 +455,23 @@ int qcfg_quant_error_sweep(qcfg_ctx* ctx, const float* const* w_dev, const int64
     if ((uintptr_t)w_dev[t] % 4) return set_error(c, QCFG_EALIGN, "sweep: tensor %d is not 4-byte aligned", t);
   }
   return launch_sweep(c, w_dev, rows, cols, n_tensors, granularity, b_lo, b_hi, sse_dev, absmax_dev, (cudaStream_t)stream);
+}
+
+int qcfg_quant_error_sweep_static(qcfg_ctx* ctx, const float* const* w_dev, const int64_t* rows, const int64_t* cols,
+                                  int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse_dev,
+                                  float* absmax_dev, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (n_tensors < 0 || !sse_dev || !absmax_dev || (n_tensors > 0 && (!w_dev || !rows || !cols)))
+    return set_error(c, QCFG_EINVAL, "static sweep: null pointer or negative count");
+  if (!bits_int(b_lo) || !bits_int(b_hi) || b_lo > b_hi) return set_error(c, QCFG_EBITS, "static sweep: bit range must lie in 2..8");
+  if (granularity != QCFG_PER_TENSOR && granularity != QCFG_PER_ROW) return set_error(c, QCFG_EINVAL, "static sweep: bad granularity");
+  for (int t = 0; t < n_tensors; ++t) {
+    if (rows[t] < 0 || cols[t] < 0 || cols[t] > 0x7fffffff) return set_error(c, QCFG_ESHAPE, "static sweep: tensor %d has a bad shape", t);
+    if (rows[t] * cols[t] > 0 && !w_dev[t]) return set_error(c, QCFG_EINVAL, "static sweep: tensor %d is null", t);
+    if ((uintptr_t)w_dev[t] % 4) return set_error(c, QCFG_EALIGN, "static sweep: tensor %d is not 4-byte aligned", t);
+  }
+  return launch_sweep_static(c, w_dev, rows, cols, n_tensors, granularity, b_lo, b_hi, sse_dev, absmax_dev, (cudaStream_t)stream);
 }
 
 int qcfg_gemm_i8(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t* qw_dev, int64_t ldw, int64_t m,

@@ -20,6 +20,7 @@ int set_error(Ctx* ctx, int code, const char* fmt, ...);
 int check_cuda(Ctx* ctx, cudaError_t e, const char* what);
 unsigned* err_word(Ctx* ctx);
 int sm_count(Ctx* ctx);
+int device_of(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);
 // optional per-launch timing of one kernel class (0 = int8 GEMM, 1 = bf16 GEMM) with CUDA events
@@ -40,6 +41,10 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
 int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
                  int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse,
                  float* absmax, cudaStream_t st);
+
+int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
+                        int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse,
+                        float* absmax, cudaStream_t st);
 
 // ----- gemm.cu ------------------------------------------------------------------------
 constexpr int kMaxSlots = 3;

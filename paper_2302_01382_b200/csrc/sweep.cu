@@ -344,4 +344,145 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
   return check_cuda(ctx, cudaGetLastError(), "sweep finalize launch");
 }
 
+
+// ------------------------------------------------------------------ sweep without allocation
+//
+// Same sweep, for callers that must not allocate device memory at call time: the block
+// partials and the descriptor tables live in a fixed device array that is part of the loaded
+// library image (about 1.05 MiB on every GPU that loads the library, until the process exits).
+
+constexpr int kStaticMaxItems = 16384;     // work items (blocks) per call: 32 Ki elements each
+constexpr int kStaticMaxTensors = 1024;
+
+struct StaticSweepScratch {
+  double partial[kStaticMaxItems * 8];
+  SweepDesc descs[kStaticMaxTensors];
+  TensorItems items[kStaticMaxTensors];
+};
+
+static __device__ __align__(256) unsigned char g_static_sweep_scratch[sizeof(StaticSweepScratch)];
+
+// Device address of the array above, per device ordinal.  In host code the array's name is only a
+// handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress, asked
+// once per device while that device is current.
+constexpr int kMaxDevices = 64;
+static void* g_static_sweep_addr[kMaxDevices] = {nullptr};
+
+int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
+                        int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse, float* absmax,
+                        cudaStream_t st) {
+  const int nb = b_hi - b_lo + 1;
+  const int per_tensor = granularity == QCFG_PER_TENSOR;
+  if (n_tensors == 0) return QCFG_OK;
+  if (n_tensors > kStaticMaxTensors)
+    return set_error(ctx, QCFG_ENOMEM, "static sweep: %d tensors exceed the fixed scratch (at most %d per call)",
+                     n_tensors, kStaticMaxTensors);
+
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "static sweep: cudaGetDevice");
+  if (dev != device_of(ctx) || dev < 0 || dev >= kMaxDevices)
+    return set_error(ctx, QCFG_ESTATE, "static sweep: the context's device (%d) must be the current device (%d)",
+                     device_of(ctx), dev);
+  if (!g_static_sweep_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_sweep_scratch);
+    if (e != cudaSuccess || !p) return check_cuda(ctx, e == cudaSuccess ? cudaErrorInvalidSymbol : e, "static sweep: cudaGetSymbolAddress");
+    g_static_sweep_addr[dev] = p;
+  }
+  StaticSweepScratch* S = static_cast<StaticSweepScratch*>(g_static_sweep_addr[dev]);
+
+  // Plan on the stack: descriptor and kernel class per tensor, then descriptors ordered by class.
+  SweepDesc plan[kStaticMaxTensors];
+  unsigned char cls_of[kStaticMaxTensors];
+  int class_count[9] = {0};
+  for (int t = 0; t < n_tensors; ++t) {
+    SweepDesc d{};
+    d.w = w[t]; d.rows = rows[t]; d.cols = (int32_t)cols[t]; d.tensor = t;
+    int cls = 0;
+    const bool vec = ((uintptr_t)w[t] % 16 == 0) && (cols[t] % 4 == 0) && cols[t] <= 8192 && cols[t] > 0;
+    if (vec) {
+      int64_t c4 = cols[t] / 4;
+      int tl = 0;
+      while (tl < 3 && c4 > (int64_t)(32 << tl) * 8) ++tl;
+      d.team_log2 = tl;
+      cls = (int)((c4 + (32 << tl) - 1) / (32 << tl));
+    }
+    int64_t rpi = cols[t] > 0 ? kItemFloats / cols[t] : 1;
+    if (cls > 0) {
+      int nteams = kThreads / (32 << d.team_log2);
+      rpi = (rpi / nteams) * nteams;
+      if (rpi < nteams) rpi = nteams;
+    }
+    if (rpi < 1) rpi = 1;
+    d.rows_per_item = (int32_t)rpi;
+    plan[t] = d;
+    cls_of[t] = (unsigned char)cls;
+    class_count[cls]++;
+  }
+  int group_desc0[9], fill[9];
+  for (int c = 0, acc = 0; c < 9; ++c) { group_desc0[c] = acc; fill[c] = acc; acc += class_count[c]; }
+  SweepDesc flat[kStaticMaxTensors];
+  for (int t = 0; t < n_tensors; ++t) flat[fill[cls_of[t]]++] = plan[t];
+
+  TensorItems titems[kStaticMaxTensors];
+  int group_item0[9], group_items[9];
+  int64_t total_items = 0;
+  for (int c = 0; c < 9; ++c) {
+    group_item0[c] = (int)total_items;
+    int64_t local = 0;
+    for (int i = 0; i < class_count[c]; ++i) {
+      SweepDesc& d = flat[group_desc0[c] + i];
+      int64_t n = (d.rows + d.rows_per_item - 1) / d.rows_per_item;
+      if (total_items + local + n > kStaticMaxItems)
+        return set_error(ctx, QCFG_ENOMEM,
+                         "static sweep: the tensors need more than %d work items of %d elements; "
+                         "split the call or use qcfg_quant_error_sweep", kStaticMaxItems, kItemFloats);
+      d.item0 = (int32_t)local;
+      titems[d.tensor].item0 = (int32_t)(total_items + local);
+      titems[d.tensor].item1 = (int32_t)(total_items + local + n);
+      local += n;
+    }
+    group_items[c] = (int)local;
+    total_items += local;
+  }
+
+  // Every block overwrites all 8 slots of its own partial entry and the finalize kernel reads only
+  // the entries of this call, so nothing left in the array by an earlier call needs clearing.
+  e = cudaMemcpyAsync(S->descs, flat, (size_t)n_tensors * sizeof(SweepDesc), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(S->items, titems, (size_t)n_tensors * sizeof(TensorItems), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "static sweep: descriptor upload");
+
+  if (per_tensor) {
+    for (int t = 0; t < n_tensors; ++t) {
+      int rc = launch_absmax(ctx, w[t], rows[t], cols[t], cols[t], QCFG_PER_TENSOR, absmax + t, st);
+      if (rc != QCFG_OK) return rc;
+    }
+  }
+  const int jlo = b_lo - 2, jhi = b_hi - 2;
+  for (int c = 0; c < 9; ++c) {
+    if (group_items[c] == 0) continue;
+    const SweepDesc* d = S->descs + group_desc0[c];
+    const int n = class_count[c];
+    double* part = S->partial + (int64_t)group_item0[c] * 8;
+    switch (c) {
+      case 0: sweep_generic_kernel<<<group_items[c], kThreads, 0, st>>>(d, n, per_tensor, absmax, jlo, jhi, part); break;
+      case 1: launch_rows<1>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 2: launch_rows<2>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 3: launch_rows<3>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 4: launch_rows<4>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 5: launch_rows<5>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 6: launch_rows<6>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      case 7: launch_rows<7>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+      default: launch_rows<8>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
+    }
+    count_launch(ctx);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return check_cuda(ctx, e, "static sweep launch");
+  }
+  sweep_finalize_kernel<<<n_tensors, 32, 0, st>>>(S->partial, S->items, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "static sweep finalize launch");
+}
+
 }  // namespace qcfg
