@@ -16,6 +16,8 @@
 // leaves through the normal teardown (TMEM is freed).
 #include <cuda.h>
 
+#include <cstring>
+
 #include "common.cuh"
 
 namespace qcfg {
@@ -34,17 +36,27 @@ constexpr int kSmemHeader = 1024;     // barriers and bookkeeping
 constexpr int kSmemMax = 232448;      // 227 KB
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
+constexpr int kNumOuts = 2 + kMaxSlots;   // raw accumulators, fp32 output, consumer code slots
+constexpr int kEpiStageBytes = 4096;      // per epilogue warp: one 32 x 128-byte piece
+
+struct OutDesc {
+  int32_t kind;       // 0 none, 1 int8 codes, 2 bf16 codes, 3 fp32, 4 int32
+  int32_t tma;        // 1: staged through shared memory and written by a TMA store
+  void* ptr;
+  int64_t ld;         // elements
+  float inv_scale, qmax;
+};
+struct OutMaps { CUtensorMap m[kNumOuts]; };
+
 struct GemmParams {
   int32_t m, n, k_blocks, bn, tiles_m, tiles_n, stages, is_bf16;
   uint32_t idesc;
   float scale_x;
   const float* scale_w;
   int32_t act;
-  float* y; int64_t ldy;
   const float* residual; int64_t ldr;
-  int32_t* acc;
   int32_t need_y;             // anything besides raw accumulators to produce
-  CodeSlot slots[kMaxSlots];
+  OutDesc outs[kNumOuts];     // [0] raw accumulators, [1] fp32 output, [2..] consumer codes
   unsigned* err;
 };
 
@@ -148,17 +160,19 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 
 // ---------------------------------------------------------------------------- epilogue math
 
+// tanh-GELU as y / (1 + exp(-2u)), u = sqrt(2/pi) (y + 0.044715 y^3), which equals
+// 0.5 y (1 + tanh u).  exp(-2u) = 2^(y (c1 + c3 y^2)) with the constants folded; one ex2 and
+// one reciprocal on the special-function unit, five FMA-pipe operations.
 __device__ __forceinline__ float gelu_tanh(float y) {
-  // y / (1 + exp(-2u)), u = sqrt(2/pi) (y + 0.044715 y^3): equals 0.5 y (1 + tanh u)
+  const float c1 = -2.302208198f;            // -2 sqrt(2/pi) log2(e)
+  const float c3 = -0.1029432396f;           // c1 * 0.044715
   float y2 = y * y;
-  float u = 0.7978845608028654f * fmaf(0.044715f * y2, y, y);
-  float e = expf(-2.0f * u);
-  return y / (1.0f + e);
-}
-__device__ __forceinline__ float apply_act(float y, int act) {
-  if (act == QCFG_ACT_RELU) return fmaxf(y, 0.0f);
-  if (act == QCFG_ACT_GELU_TANH) return gelu_tanh(y);
-  return y;
+  float t = y * fmaf(c3, y2, c1);
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return y * r;
 }
 // int8 code of Eq. 1 in the low byte: clamp, then add 1.5*2^23 (round-half-even at integer
 // granularity); the low mantissa byte is the two's-complement code.
@@ -168,27 +182,70 @@ __device__ __forceinline__ uint32_t code_byte(float y, float inv_scale, float qm
   return __float_as_uint(__fadd_rn(t, 12582912.0f)) & 0xffu;
 }
 
-// One 32-column chunk of one accumulator row.
-template <bool BF16>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, uint32_t (&v)[32], int64_t row, int col0) {
-  const bool row_ok = row < p.m;
-  const int ncols = p.n - col0;                    // valid columns in this chunk (may be <= 0 or > 32)
-  if (!row_ok || ncols <= 0) return;
-  const bool full = ncols >= 32;
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 
-  if (!BF16 && p.acc) {
-    int32_t* dst = p.acc + row * (int64_t)p.n + col0;
-    if (full && (p.n & 3) == 0) {
+// Writes one warp's 32-row x 32-column piece of an output.  Each thread holds its row's 32
+// elements packed into WORDS 32-bit words (32: fp32 / int32, 16: bf16, 8: int8).
+// Staged path: the warp lays the piece out in its 4 KB shared-memory buffer (128-byte rows use
+// the 128B swizzle so the 16-byte writes spread over all banks) and one lane issues a TMA store,
+// which writes whole rows and clips at the matrix edge.  Direct path (outputs whose row pitch is
+// not a multiple of 16 bytes): per-thread stores.
+template <int WORDS>
+__device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap* map, const uint32_t (&w)[WORDS],
+                                            bool row_ok, int ncols, int64_t row, int row0, int col0,
+                                            uint32_t stage, int lane) {
+  constexpr int kRowBytes = WORDS * 4;
+  constexpr int kElemBytes = kRowBytes / 32;
+  if (o.tma) {
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // buffer free again
+    __syncwarp();
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        reinterpret_cast<uint4*>(dst)[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    } else {
+    for (int j = 0; j < WORDS / 4; ++j) {
+      const int jj = (WORDS == 32) ? (j ^ (lane & 7)) : j;
+      st_shared_v4(stage + lane * kRowBytes + jj * 16, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) tma_store_2d(map, stage, col0, row0);
+    return;
+  }
+  if (!row_ok) return;
+  uint8_t* dst = reinterpret_cast<uint8_t*>(o.ptr) + (row * o.ld + col0) * kElemBytes;
+  if (ncols >= 32 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) if (i < ncols) dst[i] = (int32_t)v[i];
+    for (int j = 0; j < WORDS / 4; ++j)
+      reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if (i < ncols) {
+        if (kElemBytes == 4) reinterpret_cast<uint32_t*>(dst)[i] = w[i * WORDS / 32];
+        else if (kElemBytes == 2) reinterpret_cast<uint16_t*>(dst)[i] = (uint16_t)(w[i >> 1] >> (16 * (i & 1)));
+        else dst[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+      }
     }
   }
+}
 
+// One 32-column chunk of one accumulator row (all 32 lanes of the warp call this together).
+template <bool BF16>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMaps& om, uint32_t (&v)[32], int64_t row,
+                                               int row0, int col0, uint32_t stage, int lane) {
+  const int ncols = p.n - col0;                    // valid columns in this chunk (may be <= 0 or > 32)
+  if (ncols <= 0 || row0 >= p.m) return;           // warp-uniform: the piece lies outside the matrix
+  const bool row_ok = row < p.m;
+  const bool full = ncols >= 32;
+
+  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &om.m[0], v, row_ok, ncols, row, row0, col0, stage, lane);
   if (!p.need_y) return;
+
   float y[32];
   if (BF16) {
 #pragma unroll
@@ -212,7 +269,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, uint32_t (&v
       }
     }
   }
-  if (p.residual) {
+  if (p.residual && row_ok) {
     const float* r = p.residual + row * p.ldr + col0;
     if (full && (p.ldr & 3) == 0 && (((uintptr_t)p.residual) & 15) == 0) {
 #pragma unroll
@@ -228,56 +285,38 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, uint32_t (&v
       for (int i = 0; i < 32; ++i) if (i < ncols) y[i] = __fadd_rn(y[i], __ldg(r + i));
     }
   }
-  if (p.act != QCFG_ACT_NONE) {
+  if (p.act == QCFG_ACT_RELU) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) y[i] = apply_act(y[i], p.act);
+    for (int i = 0; i < 32; ++i) y[i] = fmaxf(y[i], 0.0f);
+  } else if (p.act == QCFG_ACT_GELU_TANH) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = gelu_tanh(y[i]);
   }
-  if (p.y) {
-    float* dst = p.y + row * p.ldy + col0;
-    if (full && (p.ldy & 3) == 0 && (((uintptr_t)p.y) & 15) == 0) {
+  if (p.outs[1].kind) {
+    uint32_t w[32];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        reinterpret_cast<float4*>(dst)[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) if (i < ncols) dst[i] = y[i];
-    }
+    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(y[i]);
+    store_piece<32>(p.outs[1], &om.m[1], w, row_ok, ncols, row, row0, col0, stage, lane);
   }
 #pragma unroll
   for (int s = 0; s < kMaxSlots; ++s) {
-    const CodeSlot& sl = p.slots[s];
-    if (sl.kind == 1) {
-      int8_t* dst = reinterpret_cast<int8_t*>(sl.ptr) + row * sl.ld + col0;
+    const OutDesc& o = p.outs[2 + s];
+    if (o.kind == 1) {
       uint32_t w[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        w[i] = code_byte(y[4 * i], sl.inv_scale, sl.qmax) | (code_byte(y[4 * i + 1], sl.inv_scale, sl.qmax) << 8) |
-               (code_byte(y[4 * i + 2], sl.inv_scale, sl.qmax) << 16) | (code_byte(y[4 * i + 3], sl.inv_scale, sl.qmax) << 24);
+        w[i] = code_byte(y[4 * i], o.inv_scale, o.qmax) | (code_byte(y[4 * i + 1], o.inv_scale, o.qmax) << 8) |
+               (code_byte(y[4 * i + 2], o.inv_scale, o.qmax) << 16) | (code_byte(y[4 * i + 3], o.inv_scale, o.qmax) << 24);
       }
-      if (full) {   // ld is a multiple of 16 and col0 of 32: 16-byte aligned
-        reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-      } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) if (i < ncols) dst[i] = (int8_t)((w[i >> 2] >> (8 * (i & 3))) & 0xff);
-      }
-    } else if (sl.kind == 2) {
-      __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(sl.ptr) + row * sl.ld + col0;
+      store_piece<8>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, lane);
+    } else if (o.kind == 2) {
       uint32_t w[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         __nv_bfloat162 h = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
         w[i] = *reinterpret_cast<uint32_t*>(&h);
       }
-      if (full) {   // ld is a multiple of 8 elements and col0 of 32: 16-byte aligned
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-      } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i < ncols) reinterpret_cast<uint16_t*>(dst)[i] = (uint16_t)((w[i >> 1] >> (16 * (i & 1))) & 0xffff);
-      }
+      store_piece<16>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, lane);
     }
   }
 }
@@ -287,14 +326,15 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, uint32_t (&v
 template <bool BF16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ GemmParams p) {
+            const __grid_constant__ OutMaps omaps, const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the 128B swizzle atoms
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);           // full[8] empty[8] tfull[2] tempty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
-  uint8_t* stage_base = smem + kSmemHeader;
+  uint8_t* epi_stage = smem + kSmemHeader;                       // 8 x 4 KB, 1024-aligned
+  uint8_t* stage_base = epi_stage + kEpiWarps * kEpiStageBytes;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -375,8 +415,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // ------------------------------------------------------------------ epilogue
     const int ew = warp - 2;
     const int quad = warp & 3;                 // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
-    const int half = ew >> 2;                  // interleave 32-column chunks between the two warp sets
+    const int half = ew >> 2;                  // each warp set takes a contiguous half of the tile's columns
     const int chunks = p.bn >> 5;
+    const int c_begin = chunks >= 2 ? half * (chunks >> 1) : 0;
+    const int c_end = chunks >= 2 ? c_begin + (chunks >> 1) : (half == 0 ? 1 : 0);
+    const uint32_t stage = smem_u32(epi_stage + ew * kEpiStageBytes);
     bool ok = true;
     int t = 0;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
@@ -384,16 +427,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
       if (!mbar_wait(tfull0 + 8 * a, (t >> 1) & 1, abort_flag, p.err)) { ok = false; break; }
       tc_fence_after();
-      const int64_t row = (int64_t)tm * BM + quad * 32 + lane;
-      for (int c = half; c < chunks; c += 2) {
+      const int row0 = tm * BM + quad * 32;
+      for (int c = c_begin; c < c_end; ++c) {
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * kAccCols + c * 32), v);
-        epilogue_chunk<BF16>(p, v, row, tn * p.bn + c * 32);
+        epilogue_chunk<BF16>(p, omaps, v, (int64_t)row0 + lane, row0, tn * p.bn + c * 32, stage, lane);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8 * a);
     }
+    // all TMA stores of this warp must have completed before the CTA's shared memory goes away
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   tc_fence_before();
@@ -423,6 +468,27 @@ int make_map(Ctx* ctx, CUtensorMap* map, const void* ptr, int is_bf16, int64_t k
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return set_error(ctx, QCFG_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
   return QCFG_OK;
+}
+
+// Tensor map of an output matrix [m x n] for stores of 32 x 32-element pieces.  Returns false
+// (direct stores are used instead) when the pointer or the row pitch is not 16-byte aligned.
+bool make_out_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
+  int esz; CUtensorMapDataType dt;
+  switch (o.kind) {
+    case 1: esz = 1; dt = CU_TENSOR_MAP_DATA_TYPE_UINT8; break;
+    case 2: esz = 2; dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16; break;
+    case 3: esz = 4; dt = CU_TENSOR_MAP_DATA_TYPE_FLOAT32; break;
+    default: esz = 4; dt = CU_TENSOR_MAP_DATA_TYPE_INT32; break;
+  }
+  if (((uintptr_t)o.ptr & 15) || ((o.ld * esz) & 15)) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)m};
+  cuuint64_t strides[1] = {(cuuint64_t)(o.ld * esz)};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, dt, 2, o.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        esz == 4 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -459,7 +525,7 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   p.tiles_m = (int32_t)((g.m + BM - 1) / BM);
   p.tiles_n = (int32_t)((g.n + bn - 1) / bn);
   const int stage_bytes = (BM + bn) * kStageKBytes;
-  int stages = (kSmemMax - kSmemHeader - 1024) / stage_bytes;
+  int stages = (kSmemMax - kSmemHeader - 1024 - kEpiWarps * kEpiStageBytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   p.stages = stages;
   p.is_bf16 = g.is_bf16;
@@ -467,12 +533,24 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   // at bits 7 and 10, both operands K-major, N/8 at bit 17, M/16 at bit 24
   p.idesc = ((g.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
   p.scale_x = g.scale_x; p.scale_w = g.scale_w; p.act = g.act;
-  p.y = g.y; p.ldy = g.ldy; p.residual = g.residual; p.ldr = g.ldr; p.acc = g.acc;
+  p.residual = g.residual; p.ldr = g.ldr;
+  if (g.acc && !g.is_bf16) { p.outs[0].kind = 4; p.outs[0].ptr = g.acc; p.outs[0].ld = g.n; }
+  if (g.y) { p.outs[1].kind = 3; p.outs[1].ptr = g.y; p.outs[1].ld = g.ldy; }
   p.need_y = g.y != nullptr;
-  for (int s = 0; s < kMaxSlots; ++s) { p.slots[s] = g.slots[s]; if (g.slots[s].kind) p.need_y = 1; }
-  if (!p.need_y && !g.acc) return set_error(ctx, QCFG_EINVAL, "gemm: no output requested");
+  for (int s = 0; s < kMaxSlots; ++s) {
+    if (!g.slots[s].kind) continue;
+    OutDesc& o = p.outs[2 + s];
+    o.kind = g.slots[s].kind; o.ptr = g.slots[s].ptr; o.ld = g.slots[s].ld;
+    o.inv_scale = g.slots[s].inv_scale; o.qmax = g.slots[s].qmax;
+    p.need_y = 1;
+  }
+  if (!p.need_y && !p.outs[0].kind) return set_error(ctx, QCFG_EINVAL, "gemm: no output requested");
   if (p.need_y && !g.is_bf16 && !g.scale_w) return set_error(ctx, QCFG_EINVAL, "gemm: scale_w is null");
   p.err = err_word(ctx);
+  OutMaps om;
+  memset(&om, 0, sizeof(om));
+  for (int i = 0; i < kNumOuts; ++i)
+    if (p.outs[i].kind) p.outs[i].tma = make_out_map(&om.m[i], p.outs[i], g.m, g.n) ? 1 : 0;
 
   CUtensorMap ma, mb;
   int rc = make_map(ctx, &ma, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
@@ -482,10 +560,10 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   const int num_tiles = p.tiles_m * p.tiles_n;
   int grid = sm_count(ctx);
   if (grid > num_tiles) grid = num_tiles;
-  const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)stages * stage_bytes;
+  const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)kEpiWarps * kEpiStageBytes + (size_t)stages * stage_bytes;
   prof_begin(ctx, g.is_bf16 ? 1 : 0, st);
-  if (g.is_bf16) gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(ma, mb, p);
-  else gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(ma, mb, p);
+  if (g.is_bf16) gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(ma, mb, om, p);
+  else gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(ma, mb, om, p);
   prof_end(ctx, g.is_bf16 ? 1 : 0, 2.0 * (double)g.m * (double)g.n * (double)g.k, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "gemm launch");
