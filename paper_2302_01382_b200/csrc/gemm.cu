@@ -3,13 +3,13 @@
 // activation / re-quantize epilogue fused in (Eq. 1's rescale 2^-(b-1)*gamma for both operands;
 // the "Evaluate f(x, w)" step of Algorithms 1 and 2).
 //
-// Structure (one persistent CTA per SM, 320 threads):
+// Structure (one persistent CTA per SM, 576 threads):
 //   warp 0      TMA producer: 128-byte-swizzled K-major tiles of A [128 x 128 B] and
 //               B [BN x 128 B] into a ring of shared-memory stages (mbarrier full/empty).
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=32 B per instruction)
 //               from shared-memory descriptors into one of two TMEM accumulator buffers
 //               (2 x 256 columns), and commits stage-release / accumulator-ready barriers.
-//   warps 2..9  epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns per
+//   warps 2..17 epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns per
 //               load), rescale, shortcut add, activation, stores of fp32 and/or the consumer's
 //               int8 / bf16 codes; overlaps the next tile's main loop.
 // Every mbarrier wait is bounded: after ~2 s it sets the context's error word and the CTA
@@ -27,7 +27,7 @@ namespace {
 constexpr int BM = 128;               // rows per tile (UMMA M, cta_group::1)
 constexpr int kStageKBytes = 128;     // bytes of K per stage row = one 128B swizzle atom
 constexpr int kUmmaKBytes = 32;       // bytes of K per tcgen05.mma
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;         // columns per accumulator buffer
@@ -37,7 +37,7 @@ constexpr int kSmemMax = 232448;      // 227 KB
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 constexpr int kNumOuts = 2 + kMaxSlots;   // raw accumulators, fp32 output, consumer code slots
-constexpr int kEpiStageBytes = 4096;      // per epilogue warp: one 32 x 128-byte piece
+constexpr int kEpiStageMax = 4096;        // per epilogue warp: one 32 x 128-byte piece, or two 1 KB code pieces
 
 struct OutDesc {
   int32_t kind;       // 0 none, 1 int8 codes, 2 bf16 codes, 3 fp32, 4 int32
@@ -50,6 +50,7 @@ struct OutMaps { CUtensorMap m[kNumOuts]; };
 
 struct GemmParams {
   int32_t m, n, k_blocks, bn, tiles_m, tiles_n, stages, is_bf16;
+  int32_t epi_bytes;          // staging bytes per epilogue warp (2048 or 4096)
   uint32_t idesc;
   float scale_x;
   const float* scale_w;
@@ -133,7 +134,7 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
   }
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -143,8 +144,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
         "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128B swizzle, groups of 8
 // rows 1024 bytes apart (the layout a 128B-swizzled TMA box produces).
@@ -174,12 +175,16 @@ __device__ __forceinline__ float gelu_tanh(float y) {
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
   return y * r;
 }
-// int8 code of Eq. 1 in the low byte: clamp, then add 1.5*2^23 (round-half-even at integer
-// granularity); the low mantissa byte is the two's-complement code.
-__device__ __forceinline__ uint32_t code_byte(float y, float inv_scale, float qmax) {
+// int8 code of Eq. 1 in the low byte of the returned word: clamp, then add 1.5*2^23 (a
+// round-half-even at integer granularity); the low mantissa byte is the two's-complement code.
+__device__ __forceinline__ uint32_t code_word(float y, float inv_scale, float qmax) {
   float t = __fmul_rn(y, inv_scale);
   t = fminf(fmaxf(t, -qmax), qmax);
-  return __float_as_uint(__fadd_rn(t, 12582912.0f)) & 0xffu;
+  return __float_as_uint(__fadd_rn(t, 12582912.0f));
+}
+// low bytes of four words -> one word (byte i from word i)
+__device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
 }
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int32_t x, int32_t y) {
@@ -200,20 +205,28 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 template <int WORDS>
 __device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap* map, const uint32_t (&w)[WORDS],
                                             bool row_ok, int ncols, int64_t row, int row0, int col0,
-                                            uint32_t stage, int lane) {
+                                            uint32_t stage, uint32_t stage_bytes, uint32_t& cursor, int lane) {
   constexpr int kRowBytes = WORDS * 4;
   constexpr int kElemBytes = kRowBytes / 32;
+  constexpr int kPieceBytes = 32 * kRowBytes;
   if (o.tma) {
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // buffer free again
-    __syncwarp();
+    // Pieces fill the warp's buffer one after the other; when the next one does not fit,
+    // wait until the TMA engine has read everything issued so far and start over.
+    if (cursor + kPieceBytes > stage_bytes) {
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();
+      cursor = 0;
+    }
+    const uint32_t base = stage + cursor;      // 1 KB-aligned: piece sizes are 1, 2 or 4 KB
+    cursor += kPieceBytes;
 #pragma unroll
     for (int j = 0; j < WORDS / 4; ++j) {
       const int jj = (WORDS == 32) ? (j ^ (lane & 7)) : j;
-      st_shared_v4(stage + lane * kRowBytes + jj * 16, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+      st_shared_v4(base + lane * kRowBytes + jj * 16, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0) tma_store_2d(map, stage, col0, row0);
+    if (lane == 0) tma_store_2d(map, base, col0, row0);
     return;
   }
   if (!row_ok) return;
@@ -236,14 +249,14 @@ __device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap*
 
 // One 32-column chunk of one accumulator row (all 32 lanes of the warp call this together).
 template <bool BF16>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMaps& om, uint32_t (&v)[32], int64_t row,
-                                               int row0, int col0, uint32_t stage, int lane) {
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMaps& om, uint32_t (&v)[32], float cs_lane,
+                                               int64_t row, int row0, int col0, uint32_t stage, uint32_t& cursor, int lane) {
   const int ncols = p.n - col0;                    // valid columns in this chunk (may be <= 0 or > 32)
   if (ncols <= 0 || row0 >= p.m) return;           // warp-uniform: the piece lies outside the matrix
   const bool row_ok = row < p.m;
   const bool full = ncols >= 32;
 
-  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &om.m[0], v, row_ok, ncols, row, row0, col0, stage, lane);
+  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &om.m[0], v, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
   if (!p.need_y) return;
 
   float y[32];
@@ -251,23 +264,10 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
 #pragma unroll
     for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
   } else {
-    const float* sw = p.scale_w + col0;
-    if (full && (((uintptr_t)sw) & 15) == 0) {
+    // lane i holds scale_x * scale_w[col0 + i] (loaded before the accumulator was ready)
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float4 s4 = __ldg(reinterpret_cast<const float4*>(sw) + i);
-        y[4 * i + 0] = __fmul_rn((float)(int32_t)v[4 * i + 0], __fmul_rn(p.scale_x, s4.x));
-        y[4 * i + 1] = __fmul_rn((float)(int32_t)v[4 * i + 1], __fmul_rn(p.scale_x, s4.y));
-        y[4 * i + 2] = __fmul_rn((float)(int32_t)v[4 * i + 2], __fmul_rn(p.scale_x, s4.z));
-        y[4 * i + 3] = __fmul_rn((float)(int32_t)v[4 * i + 3], __fmul_rn(p.scale_x, s4.w));
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        float s = (i < ncols) ? __ldg(sw + i) : 0.0f;
-        y[i] = __fmul_rn((float)(int32_t)v[i], __fmul_rn(p.scale_x, s));
-      }
-    }
+    for (int i = 0; i < 32; ++i)
+      y[i] = __fmul_rn((float)(int32_t)v[i], __shfl_sync(0xffffffffu, cs_lane, i));
   }
   if (p.residual && row_ok) {
     const float* r = p.residual + row * p.ldr + col0;
@@ -296,7 +296,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
     uint32_t w[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(y[i]);
-    store_piece<32>(p.outs[1], &om.m[1], w, row_ok, ncols, row, row0, col0, stage, lane);
+    store_piece<32>(p.outs[1], &om.m[1], w, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
   }
 #pragma unroll
   for (int s = 0; s < kMaxSlots; ++s) {
@@ -304,11 +304,10 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
     if (o.kind == 1) {
       uint32_t w[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        w[i] = code_byte(y[4 * i], o.inv_scale, o.qmax) | (code_byte(y[4 * i + 1], o.inv_scale, o.qmax) << 8) |
-               (code_byte(y[4 * i + 2], o.inv_scale, o.qmax) << 16) | (code_byte(y[4 * i + 3], o.inv_scale, o.qmax) << 24);
-      }
-      store_piece<8>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, lane);
+      for (int i = 0; i < 8; ++i)
+        w[i] = pack4(code_word(y[4 * i], o.inv_scale, o.qmax), code_word(y[4 * i + 1], o.inv_scale, o.qmax),
+                     code_word(y[4 * i + 2], o.inv_scale, o.qmax), code_word(y[4 * i + 3], o.inv_scale, o.qmax));
+      store_piece<8>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
     } else if (o.kind == 2) {
       uint32_t w[16];
 #pragma unroll
@@ -316,7 +315,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
         __nv_bfloat162 h = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
         w[i] = *reinterpret_cast<uint32_t*>(&h);
       }
-      store_piece<16>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, lane);
+      store_piece<16>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
     }
   }
 }
@@ -333,8 +332,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);           // full[8] empty[8] tfull[2] tempty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
-  uint8_t* epi_stage = smem + kSmemHeader;                       // 8 x 4 KB, 1024-aligned
-  uint8_t* stage_base = epi_stage + kEpiWarps * kEpiStageBytes;
+  uint8_t* epi_stage = smem + kSmemHeader;                       // kEpiWarps x epi_bytes, 1024-aligned
+  uint8_t* stage_base = epi_stage + kEpiWarps * p.epi_bytes;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -343,7 +342,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16;
   const int num_tiles = p.tiles_m * p.tiles_n;
 
+  // producer state (thread 0 only): next k-block to load
+  int ld_tile = blockIdx.x, ld_kb = 0, ld_s = 0;
+  uint32_t ld_ph = 0;
+  const int k_elems = BF16 ? kStageKBytes / 2 : kStageKBytes;
+  auto issue_load = [&]() {   // the stage's empty barrier must already have been passed
+    const int tm = ld_tile % p.tiles_m, tn = ld_tile / p.tiles_m;
+    const uint32_t a_dst = smem_u32(stage_base + (size_t)ld_s * stage_bytes);
+    mbar_expect_tx(full0 + 8 * ld_s, stage_bytes);
+    tma_load_2d(a_dst, &map_a, full0 + 8 * ld_s, ld_kb * k_elems, tm * BM);
+    tma_load_2d(a_dst + BM * kStageKBytes, &map_b, full0 + 8 * ld_s, ld_kb * k_elems, tn * p.bn);
+    if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; }
+    if (++ld_kb == p.k_blocks) { ld_kb = 0; ld_tile += gridDim.x; }
+  };
+
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, kEpiWarps); }
     *abort_flag = 0;
@@ -353,30 +368,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // Everything above touches no global memory, so under programmatic dependent launch it
+  // overlaps the tail of the previous kernel in the stream; from here on its results are needed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) {
+    // the ring is empty: fill it before the block-wide barrier so the first tiles are in flight
+    for (int i = 0; i < p.stages && ld_tile < num_tiles; ++i) issue_load();
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
-      const int k_elems = BF16 ? kStageKBytes / 2 : kStageKBytes;
-      int s = 0; uint32_t ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.err)) { ok = false; break; }
-          const uint32_t a_dst = smem_u32(stage_base + (size_t)s * stage_bytes);
-          const uint32_t b_dst = a_dst + BM * kStageKBytes;
-          mbar_expect_tx(full0 + 8 * s, stage_bytes);
-          tma_load_2d(a_dst, &map_a, full0 + 8 * s, kb * k_elems, tm * BM);
-          tma_load_2d(b_dst, &map_b, full0 + 8 * s, kb * k_elems, tn * p.bn);
-          if (++s == p.stages) { s = 0; ph ^= 1; }
-        }
+      while (ld_tile < num_tiles) {
+        if (!mbar_wait(empty0 + 8 * ld_s, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
+        issue_load();
       }
       if (!ok) {
         // give copies already in flight a bounded time to land before the CTA exits
@@ -415,27 +426,56 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // ------------------------------------------------------------------ epilogue
     const int ew = warp - 2;
     const int quad = warp & 3;                 // TMEM lanes 32*quad .. 32*quad+31 belong to this warp
-    const int half = ew >> 2;                  // each warp set takes a contiguous half of the tile's columns
+    const int colgrp = ew >> 2;                // four warp sets share the tile's columns
     const int chunks = p.bn >> 5;
-    const int c_begin = chunks >= 2 ? half * (chunks >> 1) : 0;
-    const int c_end = chunks >= 2 ? c_begin + (chunks >> 1) : (half == 0 ? 1 : 0);
-    const uint32_t stage = smem_u32(epi_stage + ew * kEpiStageBytes);
+    const int cpg = chunks >= 4 ? (chunks >> 2) : 1;
+    const int c_begin = colgrp * cpg;
+    const int c_end = c_begin < chunks ? c_begin + cpg : c_begin;
+    const uint32_t stage = smem_u32(epi_stage + ew * p.epi_bytes);
+    uint32_t cursor = 0;
     bool ok = true;
     int t = 0;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
       const int a = t & 1;
       const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+      const int row0 = tm * BM + quad * 32;
+      const int col_base = tn * p.bn + c_begin * 32;
+      // column scales of this warp's chunks, one column per lane and chunk, fetched while the
+      // tensor cores are still working on the tile
+      float cs[2] = {0.f, 0.f};
+      if (!BF16 && p.need_y) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int col = col_base + j * 32 + lane;
+          if (c_begin + j < c_end && col < p.n) cs[j] = __fmul_rn(p.scale_x, __ldg(p.scale_w + col));
+        }
+      }
       if (!mbar_wait(tfull0 + 8 * a, (t >> 1) & 1, abort_flag, p.err)) { ok = false; break; }
       tc_fence_after();
-      const int row0 = tm * BM + quad * 32;
-      for (int c = c_begin; c < c_end; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * kAccCols + c * 32), v);
-        epilogue_chunk<BF16>(p, omaps, v, (int64_t)row0 + lane, row0, tn * p.bn + c * 32, stage, lane);
+      const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * kAccCols + c_begin * 32);
+      const int nch = c_end - c_begin;           // 0, 1 or 2
+      const int64_t row = (int64_t)row0 + lane;
+      uint32_t v[32];
+      if (nch > 0) {
+        tmem_ld32_issue(tbase, v);
+        tmem_ld_wait();
+        if (nch == 1) {   // the accumulator buffer is free again once this warp's columns sit in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty0 + 8 * a);
+        }
+        epilogue_chunk<BF16>(p, omaps, v, cs[0], row, row0, col_base, stage, cursor, lane);
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * a);
+      if (nch > 1) {
+        tmem_ld32_issue(tbase + 32, v);
+        tmem_ld_wait();
+      }
+      if (nch != 1) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0 + 8 * a);
+      }
+      if (nch > 1) epilogue_chunk<BF16>(p, omaps, v, cs[1], row, row0, col_base + 32, stage, cursor, lane);
     }
     // all TMA stores of this warp must have completed before the CTA's shared memory goes away
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -525,9 +565,6 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   p.tiles_m = (int32_t)((g.m + BM - 1) / BM);
   p.tiles_n = (int32_t)((g.n + bn - 1) / bn);
   const int stage_bytes = (BM + bn) * kStageKBytes;
-  int stages = (kSmemMax - kSmemHeader - 1024 - kEpiWarps * kEpiStageBytes) / stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
-  p.stages = stages;
   p.is_bf16 = g.is_bf16;
   // instruction descriptor: D format (F32 = 1, S32 = 2) at bit 4, A/B format (BF16 = 1, S8 = 1)
   // at bits 7 and 10, both operands K-major, N/8 at bit 17, M/16 at bit 24
@@ -552,6 +589,14 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   for (int i = 0; i < kNumOuts; ++i)
     if (p.outs[i].kind) p.outs[i].tma = make_out_map(&om.m[i], p.outs[i], g.m, g.n) ? 1 : 0;
 
+  // staging per epilogue warp: two 1 KB pieces when only int8 codes are written, else one 4 KB piece
+  bool wide = false;
+  for (int i = 0; i < kNumOuts; ++i) if (p.outs[i].kind >= 2 && p.outs[i].tma) wide = true;
+  p.epi_bytes = wide ? 4096 : 2048;
+  int stages = (kSmemMax - kSmemHeader - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  p.stages = stages;
+
   CUtensorMap ma, mb;
   int rc = make_map(ctx, &ma, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
   if (rc == QCFG_OK) rc = make_map(ctx, &mb, g.b, g.is_bf16, g.k, g.n, g.ldb, bn);
@@ -560,11 +605,25 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   const int num_tiles = p.tiles_m * p.tiles_n;
   int grid = sm_count(ctx);
   if (grid > num_tiles) grid = num_tiles;
-  const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)kEpiWarps * kEpiStageBytes + (size_t)stages * stage_bytes;
+  const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)kEpiWarps * p.epi_bytes + (size_t)stages * stage_bytes;
+  // Programmatic dependent launch: the kernel's prologue (barrier set-up, TMEM allocation) may
+  // start while the previous kernel in the stream drains; it waits (griddepcontrol.wait) before
+  // touching global memory.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   prof_begin(ctx, g.is_bf16 ? 1 : 0, st);
-  if (g.is_bf16) gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(ma, mb, om, p);
-  else gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(ma, mb, om, p);
+  cudaError_t le = g.is_bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true>, ma, mb, om, p)
+                             : cudaLaunchKernelEx(&cfg, gemm_kernel<false>, ma, mb, om, p);
   prof_end(ctx, g.is_bf16 ? 1 : 0, 2.0 * (double)g.m * (double)g.n * (double)g.k, st);
+  if (le != cudaSuccess) return check_cuda(ctx, le, "gemm launch");
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "gemm launch");
 }

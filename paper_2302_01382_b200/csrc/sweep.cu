@@ -218,21 +218,31 @@ sweep_generic_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_te
 
 struct TensorItems { int32_t item0, item1; };
 
-// One warp per tensor: sums the tensor's block partials in item order.
-__global__ void sweep_finalize_kernel(const double* __restrict__ partial, const TensorItems* __restrict__ ti,
-                                      int jlo, int nb, double* __restrict__ sse, float* __restrict__ absmax,
-                                      int write_absmax) {
+// One block per tensor: 32 groups of 8 threads stride over the tensor's block partials (thread j
+// of a group owns column j: 7 sums and the maximum), then thread j < 8 combines the 32 group
+// results in a fixed order.
+__global__ void __launch_bounds__(256)
+sweep_finalize_kernel(const double* __restrict__ partial, const TensorItems* __restrict__ ti, int jlo, int nb,
+                      double* __restrict__ sse, float* __restrict__ absmax, int write_absmax) {
+  __shared__ double sm[32][8];
   const int t = blockIdx.x;
-  const int j = threadIdx.x;
+  const int j = threadIdx.x & 7, g = threadIdx.x >> 3;
   const TensorItems r = ti[t];
-  if (j < nb) {
-    double v = 0.0;
-    for (int i = r.item0; i < r.item1; ++i) v += partial[(int64_t)i * 8 + jlo + j];
-    sse[(int64_t)t * nb + j] = v;
-  } else if (j == 31 && write_absmax) {
-    double v = 0.0;
-    for (int i = r.item0; i < r.item1; ++i) v = fmax(v, partial[(int64_t)i * 8 + 7]);
-    absmax[t] = (float)v;
+  double v = 0.0;
+  for (int i = r.item0 + g; i < r.item1; i += 32) {
+    const double x = partial[(int64_t)i * 8 + j];
+    v = (j == 7) ? fmax(v, x) : v + x;
+  }
+  sm[g][j] = v;
+  __syncthreads();
+  if (threadIdx.x < 8) {
+    double a = sm[0][j];
+    for (int k = 1; k < 32; ++k) a = (j == 7) ? fmax(a, sm[k][j]) : a + sm[k][j];
+    if (j == 7) {
+      if (write_absmax) absmax[t] = (float)a;
+    } else if (j >= jlo && j < jlo + nb) {
+      sse[(int64_t)t * nb + (j - jlo)] = a;
+    }
   }
 }
 
@@ -339,7 +349,7 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
     e = cudaGetLastError();
     if (e != cudaSuccess) return check_cuda(ctx, e, "sweep launch");
   }
-  sweep_finalize_kernel<<<n_tensors, 32, 0, st>>>(partial, tidev, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
+  sweep_finalize_kernel<<<n_tensors, 256, 0, st>>>(partial, tidev, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "sweep finalize launch");
 }
@@ -480,7 +490,7 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
     e = cudaGetLastError();
     if (e != cudaSuccess) return check_cuda(ctx, e, "static sweep launch");
   }
-  sweep_finalize_kernel<<<n_tensors, 32, 0, st>>>(S->partial, S->items, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
+  sweep_finalize_kernel<<<n_tensors, 256, 0, st>>>(S->partial, S->items, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "static sweep finalize launch");
 }

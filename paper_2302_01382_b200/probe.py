@@ -1,0 +1,70 @@
+"""Small driver for profiling: a few configuration evaluations (and optionally the sweep) of a
+BERT-shaped stack with seeded synthetic inputs.
+
+    python -m paper_2302_01382_b200.probe --hidden 768 --ffn 3072 --blocks 1 --tokens 12288 --evals 3
+
+Prints host enqueue time and device time per evaluation.  Meant to be run under a profiler on
+a small case (one block is a few hundred MB at most).
+"""
+from __future__ import annotations
+
+import argparse
+import time
+
+import torch
+
+import qcfg_workloads as wl
+
+from . import Context, Model, PER_ROW
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--hidden", type=int, default=768)
+    ap.add_argument("--ffn", type=int, default=3072)
+    ap.add_argument("--blocks", type=int, default=1)
+    ap.add_argument("--tokens", type=int, default=12288)
+    ap.add_argument("--evals", type=int, default=3)
+    ap.add_argument("--bits", type=int, default=8)
+    ap.add_argument("--sweep", type=int, default=0, help="number of sweep calls to run after the evaluations")
+    ap.add_argument("--seed", type=int, default=2)
+    args = ap.parse_args()
+
+    w = wl.bert_stack(args.seed, args.tokens, args.hidden, args.ffn, args.blocks, bit_choices=None)
+    ctx = Context(0)
+    weights = [torch.from_numpy(a).cuda() for a in w.weights]
+    x = torch.from_numpy(w.x).cuda()
+    model = Model(ctx, w.layers, weights)
+    model.calibrate_model(x, w.m)
+    out = torch.empty((w.m, w.layers[-1].n_out), device="cuda")
+    ys = [None] * (len(w.layers) - 1) + [out]
+    bits = [args.bits] * len(w.layers)
+    model.eval_config(bits, x, w.m, ys)          # builds the weight-code cache
+    ctx.check_sync()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(args.evals):
+        model.eval_config(bits, x, w.m, ys)
+    e1.record()
+    t_host = time.perf_counter() - t0
+    ctx.check_sync()
+    print(f"evaluations: host enqueue {1e3 * t_host / args.evals:.3f} ms, device {e0.elapsed_time(e1) / args.evals:.3f} ms each "
+          f"({len(w.layers)} layers, {args.tokens} tokens, {args.bits} bit)")
+    if args.sweep:
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sse, amax = ctx.quant_error_sweep(weights, PER_ROW)
+        s0.record()
+        for _ in range(args.sweep):
+            ctx.quant_error_sweep(weights, PER_ROW, sse=sse, absmax=amax)
+        s1.record()
+        ctx.check_sync()
+        nbytes = 4 * sum(a.size for a in w.weights)
+        ms = s0.elapsed_time(s1) / args.sweep
+        print(f"sweep: {ms:.4f} ms per call, {nbytes / ms / 1e6:.1f} GB/s over {nbytes / 1e6:.1f} MB")
+    model.close()
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()
