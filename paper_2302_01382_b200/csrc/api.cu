@@ -126,6 +126,7 @@ struct LayerState {
   DevBuf ybuf;                     // internal fp32 output [rows x n_out]
   DevBuf abuf;                     // GEMM input codes [rows x ldk] (sized for bf16)
   DevBuf prebuf;                   // pooled fp32 input (convolution table only)
+  const float* pre_ptr = nullptr;  // pooled input actually used (may alias another layer's prebuf)
   const void* a_ptr = nullptr;     // codes actually used (may alias another layer's abuf)
   const float* y_ptr = nullptr;    // where this layer's fp32 output went (nullptr: not materialised)
   bool a_ready = false;
@@ -156,7 +157,16 @@ int64_t layer_rows(const Model* M, int l, int64_t m_ext) {
   return d.src < 0 ? m_ext : layer_rows(M, d.src, m_ext);
 }
 
-bool is_plain_linear(const qcfg_layer& d) { return d.kh == 0 && d.pool_before == QCFG_POOL_NONE; }
+// The layer's GEMM operand is its source's rows as they are (a linear layer, or a 1x1
+// convolution with stride 1 and no padding), with no pooling in between.
+bool reads_rows_directly(const qcfg_layer& d) {
+  return d.pool_before == QCFG_POOL_NONE && (d.kh == 0 || (d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0));
+}
+bool same_input(const qcfg_layer& a, const qcfg_layer& b) {
+  return a.src == b.src && a.src_col0 == b.src_col0 && a.k_in == b.k_in && a.kh == b.kh && a.kw == b.kw &&
+         a.stride == b.stride && a.pad == b.pad && a.pool_before == b.pool_before && a.in_h == b.in_h &&
+         a.in_w == b.in_w && a.in_c == b.in_c;
+}
 
 // Weight codes and per-row scales for (layer, bits); computed once and kept.
 int ensure_weight_codes(Ctx* ctx, LayerState& S, int bits, cudaStream_t st) {
@@ -199,17 +209,6 @@ int64_t ext_ld_of(const Model* M) {
   return ld;
 }
 
-// fp32 matrix a plain-linear layer reads (slice of its producer's output or of the input).
-int linear_source(Model* M, int l, const float* x_dev, Source* out) {
-  LayerState& S = M->L[l];
-  if (S.d.src < 0) { out->p = x_dev + S.d.src_col0; out->ld = S.d.k_in + 0; return QCFG_OK; }
-  LayerState& P = M->L[S.d.src];
-  if (!P.y_ptr) return set_error(M->ctx, QCFG_ESTATE, "layer %d: producer %d output not materialised", l, S.d.src);
-  out->p = P.y_ptr + S.d.src_col0;
-  out->ld = P.d.n_out;
-  return QCFG_OK;
-}
-
 // One forward pass.  calibrate = true: every layer at 16 bit, record max|input| per layer.
 int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t x_ld, int64_t m,
             float* const* y_dev, bool calibrate, cudaStream_t st) {
@@ -217,33 +216,70 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
   for (int l = 0; l < n; ++l) {
     LayerState& S = M->L[l];
     S.rows = layer_rows(M, l, m);
-    S.a_ready = false; S.a_ptr = nullptr; S.y_ptr = nullptr;
+    S.a_ready = false; S.a_ptr = nullptr; S.y_ptr = nullptr; S.pre_ptr = nullptr;
     S.bits = calibrate ? 16 : bits[l];
-    if (!is_plain_linear(S.d) || S.d.residual_from >= 0)
-      return set_error(ctx, QCFG_EUNIMPL, "layer %d: convolution / pooling / shortcut layers are not available in this build", l);
   }
   for (int l = 0; l < n; ++l) {
     LayerState& S = M->L[l];
+    const qcfg_layer& d = S.d;
     const int b = S.bits;
     int rc = ensure_weight_codes(ctx, S, b, st);
     if (rc) return rc;
 
     // ---- GEMM input codes
     if (!S.a_ready) {
-      Source src;
-      if (S.d.src < 0) { src.p = x_dev + S.d.src_col0; src.ld = x_ld; }
-      else if ((rc = linear_source(M, l, x_dev, &src))) return rc;
+      // the fp32 tensor this layer reads: [srows x sld], NHWC for the convolutional table
+      const float* sp; int64_t sld, srows;
+      if (d.src < 0) {
+        sp = x_dev; sld = x_ld;
+        srows = d.kh > 0 || d.pool_before != QCFG_POOL_NONE ? m * (int64_t)d.src_h * d.src_w : m;
+      } else {
+        LayerState& P = M->L[d.src];
+        if (!P.y_ptr) return set_error(ctx, QCFG_ESTATE, "layer %d: producer %d output not materialised", l, d.src);
+        sp = P.y_ptr; sld = P.d.n_out; srows = P.rows;
+      }
+      if (d.pool_before != QCFG_POOL_NONE) {
+        if (m * (int64_t)d.src_h * d.src_w != srows)
+          return set_error(ctx, QCFG_ESHAPE, "layer %d: source has %lld rows, src_h*src_w*m = %lld", l, (long long)srows,
+                           (long long)(m * (int64_t)d.src_h * d.src_w));
+        const int64_t prows = d.pool_before == QCFG_POOL_MAX3S2
+                                  ? m * (int64_t)((d.src_h - 1) / 2 + 1) * ((d.src_w - 1) / 2 + 1) : m;
+        for (int j = 0; j < l && !S.pre_ptr; ++j) {
+          LayerState& T = M->L[j];
+          if (T.pre_ptr && T.d.src == d.src && T.d.pool_before == d.pool_before && T.d.src_h == d.src_h && T.d.src_w == d.src_w)
+            S.pre_ptr = T.pre_ptr;
+        }
+        if (!S.pre_ptr) {
+          rc = S.prebuf.ensure(ctx, (size_t)(prows * sld) * 4);
+          if (rc) return rc;
+          if (d.pool_before == QCFG_POOL_MAX3S2)
+            rc = launch_maxpool3s2(ctx, sp, m, d.src_h, d.src_w, (int)sld, (float*)S.prebuf.p, st);
+          else
+            rc = launch_avgpool(ctx, sp, m, d.src_h * d.src_w, (int)sld, (float*)S.prebuf.p, st);
+          if (rc) return rc;
+          S.pre_ptr = (const float*)S.prebuf.p;
+        }
+        sp = S.pre_ptr; srows = prows;
+      }
+      const bool direct = d.kh == 0 || (d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0);
+      if (d.kh > 0) {
+        if (sld != d.in_c || srows != m * (int64_t)d.in_h * d.in_w)
+          return set_error(ctx, QCFG_ESHAPE, "layer %d: convolution input is [%lld x %lld], expected [%lld x %d]", l,
+                           (long long)srows, (long long)sld, (long long)(m * (int64_t)d.in_h * d.in_w), d.in_c);
+      } else if (srows != S.rows) {
+        return set_error(ctx, QCFG_ESHAPE, "layer %d: source rows %lld differ from layer rows %lld", l, (long long)srows, (long long)S.rows);
+      }
+      const int64_t width = d.kh > 0 ? d.in_c : d.k_in;       // columns of the tensor that is calibrated
+      const float* tp = sp + (d.kh > 0 ? 0 : d.src_col0);
       if (calibrate) {
-        rc = launch_absmax(ctx, src.p, S.rows, S.d.k_in, src.ld, QCFG_PER_TENSOR, (float*)M->act_absmax_dev.p + l, st);
+        rc = launch_absmax(ctx, tp, srows, width, sld, QCFG_PER_TENSOR, (float*)M->act_absmax_dev.p + l, st);
         if (rc) return rc;
       }
-      // reuse the codes of an earlier layer that reads the same slice with the same grid
+      // reuse the codes of an earlier layer that reads the same input with the same grid
       int share = -1;
       for (int j = 0; j < l && share < 0; ++j) {
         LayerState& T = M->L[j];
-        if (T.d.src == S.d.src && T.d.src_col0 == S.d.src_col0 && T.d.k_in == S.d.k_in && T.bits == b &&
-            T.a_ptr && (b == 16 || T.act_absmax == S.act_absmax))
-          share = j;
+        if (same_input(T.d, d) && T.bits == b && T.a_ptr && (b == 16 || T.act_absmax == S.act_absmax)) share = j;
       }
       if (share >= 0) {
         S.a_ptr = M->L[share].a_ptr;
@@ -252,7 +288,10 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
         if (rc) return rc;
         float sc = 1.0f, inv = 1.0f;
         if (b != 16) host_scales(S.act_absmax, b, &sc, &inv);
-        rc = launch_quantize(ctx, src.p, S.rows, S.d.k_in, src.ld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
+        if (direct)
+          rc = launch_quantize(ctx, tp, S.rows, d.k_in, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
+        else
+          rc = launch_im2col_quantize(ctx, sp, m, d.in_h, d.in_w, d.in_c, d.kh, d.kw, d.stride, d.pad, inv, b, S.abuf.p, S.ldk, st);
         if (rc) return rc;
         S.a_ptr = S.abuf.p;
       }
@@ -278,7 +317,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     for (int c : S.consumers) {
       LayerState& C = M->L[c];
       const int cb = calibrate ? 16 : bits[c];
-      const bool fusable = ctx->fuse && !calibrate && is_plain_linear(C.d) && C.d.src_col0 == 0 && C.d.k_in == S.d.n_out;
+      const bool fusable = ctx->fuse && !calibrate && reads_rows_directly(C.d) && C.d.src_col0 == 0 && C.d.k_in == S.d.n_out;
       if (!fusable) { all_fused = false; continue; }
       float csc = 1.0f, cinv = 1.0f;
       if (cb != 16) host_scales(C.act_absmax, cb, &csc, &cinv);
@@ -311,6 +350,11 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     }
     g.y = y_out; g.ldy = S.d.n_out;
     S.y_ptr = y_out;
+    if (d.residual_from >= 0) {
+      LayerState& R = M->L[d.residual_from];
+      if (!R.y_ptr || R.rows != S.rows) return set_error(ctx, QCFG_ESHAPE, "layer %d: shortcut from layer %d is unavailable or has other rows", l, d.residual_from);
+      g.residual = R.y_ptr; g.ldr = R.d.n_out;
+    }
     rc = launch_gemm(ctx, g, st);
     if (rc) return rc;
   }
@@ -518,11 +562,14 @@ int qcfg_model_create(qcfg_ctx* ctx, const qcfg_layer* layers, int32_t n_layers,
     if (d.src >= l || d.src < -1 || d.residual_from >= l || d.residual_from < -1) return set_error(c, QCFG_ESHAPE, "layer %d: src / residual_from must be earlier layers", l);
     if (d.act < QCFG_ACT_NONE || d.act > QCFG_ACT_GELU_TANH) return set_error(c, QCFG_EINVAL, "layer %d: bad activation", l);
     if (d.src_col0 < 0) return set_error(c, QCFG_ESHAPE, "layer %d: negative src_col0", l);
-    if (d.kh == 0 && d.pool_before == QCFG_POOL_NONE && d.src >= 0 && d.src_col0 + d.k_in > layers[d.src].n_out)
+    if (d.kh == 0 && d.src >= 0 && d.src_col0 + d.k_in > layers[d.src].n_out)
       return set_error(c, QCFG_ESHAPE, "layer %d: reads columns beyond its producer's output", l);
     if (d.kh > 0 && (d.kw <= 0 || d.stride <= 0 || d.pad < 0 || d.in_h <= 0 || d.in_w <= 0 || d.in_c <= 0 ||
                      (int64_t)d.kh * d.kw * d.in_c != d.k_in))
       return set_error(c, QCFG_ESHAPE, "layer %d: inconsistent convolution geometry", l);
+    if (d.pool_before != QCFG_POOL_NONE && (d.pool_before < 0 || d.pool_before > QCFG_POOL_GLOBAL_AVG || d.src_h <= 0 || d.src_w <= 0))
+      return set_error(c, QCFG_ESHAPE, "layer %d: pooling needs src_h and src_w", l);
+    if (d.kh > 0 && d.src >= 0 && layers[d.src].n_out != d.in_c) return set_error(c, QCFG_ESHAPE, "layer %d: in_c differs from its producer's width", l);
     if (d.residual_from >= 0 && layers[d.residual_from].n_out != d.n_out) return set_error(c, QCFG_ESHAPE, "layer %d: shortcut width differs", l);
   }
   qcfg_model* h = new (std::nothrow) qcfg_model();

@@ -37,6 +37,12 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
                     const float* inv_scale_ptr, float inv_scale_val, int granularity, int bits,
                     void* q, int64_t ldq, cudaStream_t st);
 
+// ----- conv.cu ------------------------------------------------------------------------
+int launch_maxpool3s2(Ctx* ctx, const float* src, int64_t B, int H, int W, int C, float* dst, cudaStream_t st);
+int launch_avgpool(Ctx* ctx, const float* src, int64_t B, int HW, int C, float* dst, cudaStream_t st);
+int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, int C, int kh, int kw, int stride,
+                           int pad, float inv_scale, int bits, void* q, int64_t ldq, cudaStream_t st);
+
 // ----- sweep.cu -----------------------------------------------------------------------
 int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
                  int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse,

@@ -174,3 +174,24 @@ def test_model_argument_errors(ctx):
         model.calibrate_model(xn, w.m)
     assert e.value.status == q.ENONFINITE
     model.close()
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+def test_resnet_small_teacher_forced(ctx, fuse):
+    """Convolutional table at reduced size: im2col operands (3-channel 7x7/2 stem, 3x3 with stride 1
+    and 2, 1x1 with stride 1 and 2), max-pool, shortcuts, global average pool, 16-bit stem and fc."""
+    ctx.set_fusion(fuse)
+    try:
+        w = wl.resnet50(seed=3, batch=3, in_hw=64, width=16, n_classes=10, blocks=(2, 1, 2, 1))
+        model, x = build(ctx, w)
+        act_g, w_amax = check_calibration(model, w)
+        for bits in (w.bits, [8] * len(w.layers)):
+            ys = run_eval(ctx, model, w, x, bits)
+            teacher_forced_check(ctx, model, w, x, bits, ys, act_g, w_amax)
+        outs = orc.eval_config(w.layers, w.weights, w.bits, w.x, list(act_g), w_amax)
+        last = host(ys[-1])
+        ref_all8 = orc.eval_config(w.layers, w.weights, [8] * len(w.layers), w.x, list(act_g), w_amax)
+        assert np.linalg.norm(last - ref_all8[-1]) <= 2e-2 * np.linalg.norm(ref_all8[-1])
+        model.close()
+    finally:
+        ctx.set_fusion(True)
