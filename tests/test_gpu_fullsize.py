@@ -123,3 +123,45 @@ def test_bert_large_x24_bisection_step(ctx):
     sampled_teacher_forced(ctx, model, w, x, seq[0], layers=set(range(0, 144, 3)))
     sampled_teacher_forced(ctx, model, w, x, seq[3], layers={0, 1, 2, 3, 4, 5, 70, 71, 142, 143})
     model.close()
+
+
+def test_resnet50_batch128_sampled_images(ctx):
+    """ResNet-50 v1.5 table at batch 128: every layer checked under teacher forcing on two whole
+    images (rows of different images are independent), from the GPU's own inputs to that layer."""
+    import paper_2302_01382_b200 as q
+    w = wl.resnet50()
+    assert len(w.layers) == 54 and w.bits[0] == 16 and w.bits[-1] == 16
+    weights = [torch.from_numpy(a).cuda() for a in w.weights]
+    x = torch.from_numpy(w.x).cuda()
+    model = q.Model(ctx, w.layers, weights)
+    model.calibrate_model(x, w.m)
+    act_g = np.array(model.act_absmax(), np.float32)
+    rows_of = [wl.layer_rows(w.layers, l, w.m) for l in range(54)]
+    ys = [torch.full((rows_of[l], lay.n_out), float("nan"), device="cuda") for l, lay in enumerate(w.layers)]
+    model.eval_config(w.bits, x, w.m, ys)
+    ctx.check_sync()
+    for img in (0, 127):
+        per = [r // w.m for r in rows_of]
+        outs = [ys[l][img * per[l]:(img + 1) * per[l]].cpu().numpy() for l in range(54)]
+        x_img = w.x[img:img + 1]
+        for l, lay in enumerate(w.layers):
+            assert np.all(np.isfinite(outs[l])), f"layer {l}: unwritten output"
+            b = int(w.bits[l])
+            xin = orc.layer_input(w.layers, l, x_img, outs)
+            res = outs[lay.residual_from] if lay.residual_from >= 0 else None
+            w_amax = orc.absmax(w.weights[l], orc.PER_ROW)
+            y_ref, taps = orc.eval_layer_teacher_forced(lay, w.weights[l], xin, b, act_g[l], w_amax, residual=res)
+            if b == 16:
+                assert np.linalg.norm(outs[l] - y_ref) <= 1e-2 * np.linalg.norm(y_ref), l
+                assert np.abs(outs[l] - y_ref).max() <= 1e-2 * np.abs(y_ref).max(), l
+                continue
+            if img == 0:      # codes and accumulators once per layer (the dumps are whole-batch buffers)
+                qx = torch.empty((rows_of[l], lay.k_in), dtype=torch.int8, device="cuda")
+                acc = torch.empty((rows_of[l], lay.n_out), dtype=torch.int32, device="cuda")
+                model.debug_dump(l, qx, None, acc)
+                ctx.check_sync()
+                np.testing.assert_array_equal(qx[:per[l]].cpu().numpy(), taps["qx"], err_msg=f"layer {l} input codes")
+                np.testing.assert_array_equal(acc[:per[l]].cpu().numpy(), taps["acc"], err_msg=f"layer {l} accumulators")
+                del qx, acc
+            np.testing.assert_array_equal(outs[l].view(np.uint32), y_ref.view(np.uint32), err_msg=f"layer {l} image {img}")
+    model.close()
