@@ -169,6 +169,17 @@ int qcfg_gemm_i8(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t*
                  const float* scale_w_dev, int act, float* y_dev, int32_t* acc_dev,
                  void* stream);
 
+/* The same GEMM with the consumer's quantize step (Eq. 1 at the consumer's bit width) fused
+ * into the epilogue, as a configuration evaluation runs it between two quantized layers:
+ * q_out = clamp(round_half_even(act(y) * next_inv_scale), +-qmax(next_bits)) as int8 for
+ * next_bits in 2..8, or bfloat16(act(y)) for next_bits == 16 (next_inv_scale ignored).  The fp32
+ * y is never written.  q_out_dev is [m x ldq] (int8 or 2-byte bfloat16), 16-byte aligned, ldq a
+ * multiple of 16 and >= n; columns n..ldq-1 are left untouched.                              */
+int qcfg_gemm_i8_requant(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t* qw_dev,
+                         int64_t ldw, int64_t m, int64_t n, int64_t k, float scale_x,
+                         const float* scale_w_dev, int act, float next_inv_scale, int next_bits,
+                         void* q_out_dev, int64_t ldq, void* stream);
+
 /* 16-bit layer (the paper's floating-point-16 baseline precision, Table 1):
  * y = act(sum_k x[m][k]*w[n][k]) with bfloat16 operands (2-byte elements, leading
  * dimensions multiples of 8 elements, padding zero) and fp32 accumulation.                */

@@ -23,7 +23,7 @@ EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT, EUNIM
 
 EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error", "qcfg_launch_count",
            "qcfg_set_fusion", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
-           "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_bf16", "qcfg_model_create",
+           "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
            "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_debug_dump"]
 
@@ -68,6 +68,7 @@ def load_library() -> C.CDLL:
         "qcfg_quant_error_sweep": [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), i32, ci, ci, ci, vp, vp, vp],
         "qcfg_quant_error_sweep_static": [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(i64), i32, ci, ci, ci, vp, vp, vp],
         "qcfg_gemm_i8": [vp, vp, i64, vp, i64, i64, i64, i64, f32, vp, ci, vp, vp, vp],
+        "qcfg_gemm_i8_requant": [vp, vp, i64, vp, i64, i64, i64, i64, f32, vp, ci, f32, ci, vp, i64, vp],
         "qcfg_gemm_bf16": [vp, vp, i64, vp, i64, i64, i64, i64, ci, vp, vp],
         "qcfg_model_create": [vp, C.POINTER(LayerStruct), i32, C.POINTER(vp)],
         "qcfg_model_destroy": [vp],
@@ -219,6 +220,16 @@ class Context:
         self._check(self.lib.qcfg_gemm_i8(self.h, _ptr(qx), qx.stride(0), _ptr(qw), qw.stride(0), m, n, k, scale_x,
                                           _ptr(scale_w), act, _ptr(y), _ptr(acc), _stream(stream)))
         return y, acc
+
+    def gemm_i8_requant(self, qx: torch.Tensor, qw: torch.Tensor, k: int, scale_x: float, scale_w: torch.Tensor, act: int,
+                        next_inv_scale: float, next_bits: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        m, n = qx.shape[0], qw.shape[0]
+        if out is None:
+            out = torch.zeros((m, (n + 15) // 16 * 16), dtype=torch.bfloat16 if next_bits == 16 else torch.int8, device=qx.device)
+        self._check(self.lib.qcfg_gemm_i8_requant(self.h, _ptr(qx), qx.stride(0), _ptr(qw), qw.stride(0), m, n, k, scale_x,
+                                                  _ptr(scale_w), act, next_inv_scale, next_bits, _ptr(out), out.stride(0),
+                                                  _stream(stream)))
+        return out
 
     def gemm_bf16(self, x: torch.Tensor, w: torch.Tensor, k: int, act: int = ACT_NONE, stream=None) -> torch.Tensor:
         m, n = x.shape[0], w.shape[0]

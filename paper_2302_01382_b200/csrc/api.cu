@@ -536,6 +536,25 @@ int qcfg_gemm_i8(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t*
   return launch_gemm(c, g, (cudaStream_t)stream);
 }
 
+int qcfg_gemm_i8_requant(qcfg_ctx* ctx, const int8_t* qx_dev, int64_t ldx, const int8_t* qw_dev, int64_t ldw, int64_t m,
+                         int64_t n, int64_t k, float scale_x, const float* scale_w_dev, int act, float next_inv_scale,
+                         int next_bits, void* q_out_dev, int64_t ldq, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  if (!qx_dev || !qw_dev || !scale_w_dev || !q_out_dev) return set_error(c, QCFG_EINVAL, "gemm_i8_requant: null pointer");
+  if (act < QCFG_ACT_NONE || act > QCFG_ACT_GELU_TANH) return set_error(c, QCFG_EINVAL, "gemm_i8_requant: bad activation");
+  if (!bits_ok(next_bits)) return set_error(c, QCFG_EBITS, "gemm_i8_requant: next_bits must be 2..8 or 16, got %d", next_bits);
+  if (ldq < n) return set_error(c, QCFG_ESHAPE, "gemm_i8_requant: ldq < n");
+  if (ldq % 16 || (uintptr_t)q_out_dev % 16 || (uintptr_t)scale_w_dev % 4) return set_error(c, QCFG_EALIGN, "gemm_i8_requant: q_out_dev must be 16-byte aligned with ldq a multiple of 16");
+  GemmArgs g{};
+  g.a = qx_dev; g.lda = ldx; g.b = qw_dev; g.ldb = ldw; g.m = m; g.n = n; g.k = k;
+  g.is_bf16 = 0; g.scale_x = scale_x; g.scale_w = scale_w_dev; g.act = act;
+  g.slots[0].ptr = q_out_dev; g.slots[0].ld = ldq; g.slots[0].inv_scale = next_inv_scale;
+  g.slots[0].qmax = next_bits == 16 ? 0.0f : qmax_of(next_bits);
+  g.slots[0].kind = next_bits == 16 ? 2 : 1;
+  return launch_gemm(c, g, (cudaStream_t)stream);
+}
+
 int qcfg_gemm_bf16(qcfg_ctx* ctx, const void* x_bf16_dev, int64_t ldx, const void* w_bf16_dev, int64_t ldw, int64_t m,
                    int64_t n, int64_t k, int act, float* y_dev, void* stream) {
   if (!ctx) return QCFG_EINVAL;

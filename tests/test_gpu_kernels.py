@@ -206,6 +206,30 @@ def test_gemm_i8_activations(ctx, act):
         np.testing.assert_allclose(host(y), ref, rtol=1e-6, atol=1e-6 * np.abs(ref).max())
 
 
+@pytest.mark.parametrize("next_bits", [2, 4, 8, 16])
+@pytest.mark.parametrize("m,n,k,act", [(300, 200, 150, 0), (1000, 768, 768, 1), (515, 1000, 256, 0), (260, 330, 144, 1)])
+def test_gemm_i8_requant_codes_bit_exact(ctx, m, n, k, act, next_bits):
+    rng = np.random.default_rng(m + n + k + next_bits)
+    ld = (k + 15) // 16 * 16
+    qx, qw = _codes(rng, m, k, ld), _codes(rng, n, k, ld)
+    sw = (10.0 ** rng.uniform(-4, -2, n)).astype(np.float32)
+    sx = np.float32(0.0173)
+    y = orc.activation(orc.dequant_output(orc.int_gemm(qx[:, :k], qw[:, :k]), sx, sw), act)
+    if next_bits == 16:
+        out = ctx.gemm_i8_requant(dev(qx), dev(qw), k, float(sx), dev(sw), act, 1.0, 16)
+        ctx.check_sync()
+        got = host(out.float())[:, :n]
+        np.testing.assert_array_equal(got.view(np.uint32), orc.bf16_round(y).view(np.uint32))
+    else:
+        A = np.float32(np.abs(y).max() * 0.6)            # calibrated maximum below the data: live clip
+        _, inv = orc.scales_from_absmax(A, next_bits)
+        out = ctx.gemm_i8_requant(dev(qx), dev(qw), k, float(sx), dev(sw), act, float(inv), next_bits)
+        ctx.check_sync()
+        want = orc.quantize(y, inv, next_bits)
+        np.testing.assert_array_equal(host(out)[:, :n], want)
+        assert np.abs(want).max() == orc.qmax(next_bits)
+
+
 @pytest.mark.parametrize("m,n,k", [(64, 16, 16), (300, 200, 150), (1000, 768, 768), (129, 1000, 3072), (128, 1000, 2048)])
 def test_gemm_bf16_matches_fp64_reference(ctx, m, n, k):
     import paper_2302_01382_b200 as q
