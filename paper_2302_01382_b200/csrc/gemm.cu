@@ -456,26 +456,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       const int nch = c_end - c_begin;           // 0, 1 or 2
       const int64_t row = (int64_t)row0 + lane;
       uint32_t v[32];
-      if (nch > 0) {
-        tmem_ld32_issue(tbase, v);
+      // one copy of the chunk code, looped: keeps the instruction footprint small
+#pragma unroll 1
+      for (int c = 0; c < nch; ++c) {
+        tmem_ld32_issue(tbase + 32 * c, v);
         tmem_ld_wait();
-        if (nch == 1) {   // the accumulator buffer is free again once this warp's columns sit in registers
+        if (c == nch - 1) {   // the accumulator buffer is free again once this warp's columns sit in registers
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(tempty0 + 8 * a);
         }
-        epilogue_chunk<BF16>(p, omaps, v, cs[0], row, row0, col_base, stage, cursor, lane);
+        epilogue_chunk<BF16>(p, omaps, v, c ? cs[1] : cs[0], row, row0, col_base + 32 * c, stage, cursor, lane);
       }
-      if (nch > 1) {
-        tmem_ld32_issue(tbase + 32, v);
-        tmem_ld_wait();
-      }
-      if (nch != 1) {
-        tc_fence_before();
+      if (nch == 0) {
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty0 + 8 * a);
       }
-      if (nch > 1) epilogue_chunk<BF16>(p, omaps, v, cs[1], row, row0, col_base + 32, stage, cursor, lane);
     }
     // all TMA stores of this warp must have completed before the CTA's shared memory goes away
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
