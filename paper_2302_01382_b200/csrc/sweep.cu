@@ -22,7 +22,19 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kNB = 7;                       // bit widths 2..8
 constexpr float kMagic = 12582912.0f;        // 1.5 * 2^23
-constexpr int kItemFloats = 32 * 1024;       // elements per work item (one block)
+constexpr int kItemFloatsMin = 8 * 1024;     // elements per work item (one block): bounds
+constexpr int kItemFloatsMax = 256 * 1024;
+
+// Work-item size for a call: about eight items per SM (two resident blocks, four rounds), so
+// that a block's start-up cost is amortised and the last round stays short.
+inline int64_t item_floats_for(const int64_t* rows, const int64_t* cols, int32_t n_tensors, int sms) {
+  int64_t total = 0;
+  for (int t = 0; t < n_tensors; ++t) total += rows[t] * cols[t];
+  int64_t f = total / ((int64_t)sms * 8);
+  if (f < kItemFloatsMin) f = kItemFloatsMin;
+  if (f > kItemFloatsMax) f = kItemFloatsMax;
+  return f;
+}
 
 struct SweepDesc {
   const float* w;
@@ -35,13 +47,17 @@ struct SweepDesc {
   int32_t pad;
 };
 
-__device__ __forceinline__ const SweepDesc& find_desc(const SweepDesc* __restrict__ d, int n, int item) {
-  int lo = 0, hi = n - 1;
-  while (lo < hi) {
-    int mid = (lo + hi + 1) >> 1;
-    if (d[mid].item0 <= item) lo = mid; else hi = mid - 1;
+// The descriptor whose item range holds `item`: every thread tests a few descriptors (one
+// round of loads instead of a dependent chain), the winner publishes its index.
+__device__ __forceinline__ SweepDesc find_desc(const SweepDesc* __restrict__ d, int n, int item) {
+  __shared__ int s_idx;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int lo = d[i].item0;
+    const int hi = (i + 1 < n) ? d[i + 1].item0 : 0x7fffffff;
+    if (lo <= item && item < hi) s_idx = i;       // exactly one i qualifies (item0 strictly increases)
   }
-  return d[lo];
+  __syncthreads();
+  return d[s_idx];
 }
 
 __device__ __forceinline__ void scales_for_lane(float A, int lane, float& s, float& inv) {
@@ -79,7 +95,18 @@ __device__ __forceinline__ void block_reduce_store(double (&dacc)[kNB], float am
   }
 }
 
-// Rows of up to 32*V*team float4; cols % 4 == 0 and 16-byte aligned rows.
+// Two elements per instruction: the four operations of one (element, b) evaluation as packed
+// fp32 arithmetic (sm_100 fma.rn.f32x2 / add.rn.f32x2), which halves the issue slots they need.
+__device__ __forceinline__ void err8(float2 x, float2 s, float2 inv, float2& acc) {
+  const float2 magic = make_float2(kMagic, kMagic), nmagic = make_float2(-kMagic, -kMagic);
+  float2 u = __ffma2_rn(x, inv, magic);
+  float2 r = __fadd2_rn(u, nmagic);
+  float2 e = __ffma2_rn(make_float2(-s.x, -s.y), r, x);
+  acc = __ffma2_rn(e, e, acc);
+}
+
+// Rows of up to 32*V*team float4; cols % 4 == 0 and 16-byte aligned rows.  All 7 bit widths are
+// always evaluated (a narrower request only selects columns in the finalize kernel).
 template <int V>
 __global__ void __launch_bounds__(kThreads, 2)
 sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tensor,
@@ -105,7 +132,6 @@ sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tenso
   for (int j = 0; j < kNB; ++j) dacc[j] = 0.0;
   float amax_blk = 0.0f;
 
-  float4 cur[V], nxt[V];
   auto load_row = [&](float4 (&dst)[V], int64_t row) {
     const float4* p = reinterpret_cast<const float4*>(d.w + row * (int64_t)d.cols);
 #pragma unroll
@@ -114,11 +140,7 @@ sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tenso
       dst[v] = (row < row1 && c < c4) ? __ldg(p + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
-  load_row(cur, row0 + team);
-
-  for (int it = 0; it < n_iter; ++it) {
-    load_row(nxt, row0 + (int64_t)(it + 1) * nteams + team);   // prefetch (zeros past the end)
-
+  auto process_row = [&](const float4 (&cur)[V]) {
     float m = 0.0f;
 #pragma unroll
     for (int v = 0; v < V; ++v)
@@ -138,29 +160,37 @@ sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tenso
 
     float s_l, inv_l;
     scales_for_lane(m, lane, s_l, inv_l);
-    float s[kNB], inv[kNB], facc[kNB];
+    float2 s[kNB], inv[kNB], facc[kNB];
 #pragma unroll
     for (int j = 0; j < kNB; ++j) {
-      s[j] = __shfl_sync(0xffffffffu, s_l, j);
-      inv[j] = __shfl_sync(0xffffffffu, inv_l, j);
-      facc[j] = 0.0f;
+      const float sj = __shfl_sync(0xffffffffu, s_l, j), ij = __shfl_sync(0xffffffffu, inv_l, j);
+      s[j] = make_float2(sj, sj);
+      inv[j] = make_float2(ij, ij);
+      facc[j] = make_float2(0.0f, 0.0f);
     }
 #pragma unroll
     for (int v = 0; v < V; ++v) {
+      const float2 lo = make_float2(cur[v].x, cur[v].y), hi = make_float2(cur[v].z, cur[v].w);
 #pragma unroll
       for (int j = 0; j < kNB; ++j) {
-        if (j >= jlo && j <= jhi) {
-          err4(cur[v].x, s[j], inv[j], facc[j]);
-          err4(cur[v].y, s[j], inv[j], facc[j]);
-          err4(cur[v].z, s[j], inv[j], facc[j]);
-          err4(cur[v].w, s[j], inv[j], facc[j]);
-        }
+        err8(lo, s[j], inv[j], facc[j]);
+        err8(hi, s[j], inv[j], facc[j]);
       }
     }
 #pragma unroll
-    for (int j = 0; j < kNB; ++j) dacc[j] += (double)facc[j];
-#pragma unroll
-    for (int v = 0; v < V; ++v) cur[v] = nxt[v];
+    for (int j = 0; j < kNB; ++j) dacc[j] += (double)(facc[j].x + facc[j].y);
+  };
+
+  // two register buffers, used alternately: the next row is in flight while this one is processed
+  float4 ra[V], rb[V];
+  load_row(ra, row0 + team);
+  for (int it = 0; it < n_iter; it += 2) {
+    load_row(rb, row0 + (int64_t)(it + 1) * nteams + team);   // zeros past the end
+    process_row(ra);
+    if (it + 1 < n_iter) {
+      load_row(ra, row0 + (int64_t)(it + 2) * nteams + team);
+      process_row(rb);
+    }
   }
   block_reduce_store(dacc, amax_blk, partial + (int64_t)blockIdx.x * 8);
 }
@@ -260,6 +290,7 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
   const int per_tensor = granularity == QCFG_PER_TENSOR;
   if (n_tensors == 0) return QCFG_OK;
 
+  const int64_t item_floats = item_floats_for(rows, cols, n_tensors, sm_count(ctx));
   // Group tensors by kernel variant: class 0 = generic, class V (1..8) = register-resident rows.
   std::vector<SweepDesc> groups[9];
   std::vector<TensorItems> titems(n_tensors);
@@ -275,7 +306,7 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
       d.team_log2 = tl;
       cls = (int)((c4 + (32 << tl) - 1) / (32 << tl));     // float4 per thread, 1..8
     }
-    int64_t rpi = cols[t] > 0 ? kItemFloats / cols[t] : 1;
+    int64_t rpi = cols[t] > 0 ? item_floats / cols[t] : 1;
     if (cls > 0) {
       int nteams = kThreads / (32 << d.team_log2);
       rpi = (rpi / nteams) * nteams;
@@ -361,7 +392,7 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
 // partials and the descriptor tables live in a fixed device array that is part of the loaded
 // library image (about 1.05 MiB on every GPU that loads the library, until the process exits).
 
-constexpr int kStaticMaxItems = 16384;     // work items (blocks) per call: 32 Ki elements each
+constexpr int kStaticMaxItems = 16384;     // work items (blocks) per call
 constexpr int kStaticMaxTensors = 1024;
 
 struct StaticSweepScratch {
@@ -402,6 +433,7 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
   }
   StaticSweepScratch* S = static_cast<StaticSweepScratch*>(g_static_sweep_addr[dev]);
 
+  const int64_t item_floats = item_floats_for(rows, cols, n_tensors, sm_count(ctx));
   // Plan on the stack: descriptor and kernel class per tensor, then descriptors ordered by class.
   SweepDesc plan[kStaticMaxTensors];
   unsigned char cls_of[kStaticMaxTensors];
@@ -418,7 +450,7 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
       d.team_log2 = tl;
       cls = (int)((c4 + (32 << tl) - 1) / (32 << tl));
     }
-    int64_t rpi = cols[t] > 0 ? kItemFloats / cols[t] : 1;
+    int64_t rpi = cols[t] > 0 ? item_floats / cols[t] : 1;
     if (cls > 0) {
       int nteams = kThreads / (32 << d.team_log2);
       rpi = (rpi / nteams) * nteams;
@@ -446,8 +478,8 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
       int64_t n = (d.rows + d.rows_per_item - 1) / d.rows_per_item;
       if (total_items + local + n > kStaticMaxItems)
         return set_error(ctx, QCFG_ENOMEM,
-                         "static sweep: the tensors need more than %d work items of %d elements; "
-                         "split the call or use qcfg_quant_error_sweep", kStaticMaxItems, kItemFloats);
+                         "static sweep: the tensors need more than %d work items (of about %lld elements each); "
+                         "split the call or use qcfg_quant_error_sweep", kStaticMaxItems, (long long)item_floats);
       d.item0 = (int32_t)local;
       titems[d.tensor].item0 = (int32_t)(total_items + local);
       titems[d.tensor].item1 = (int32_t)(total_items + local + n);
