@@ -20,6 +20,10 @@ struct Ctx {
   int64_t launches = 0;
   int fuse = 1;
   char msg[512] = {0};
+  // last sweep tables uploaded to the scratch buffer
+  const void* sweep_base = nullptr;
+  cudaStream_t sweep_stream = nullptr;
+  std::vector<char> sweep_tables;
   // per-launch event timing (off by default)
   int prof = 0;
   std::vector<cudaEvent_t> ev;      // pairs: ev[2i] before, ev[2i+1] after
@@ -74,6 +78,17 @@ int check_cuda(Ctx* ctx, cudaError_t e, const char* what) {
   if (e == cudaSuccess) return QCFG_OK;
   return set_error(ctx, e == cudaErrorMemoryAllocation ? QCFG_ENOMEM : QCFG_ECUDA, "%s: %s", what, cudaGetErrorString(e));
 }
+bool sweep_tables_cached(Ctx* ctx, const void* dev_base, cudaStream_t st, const void* a, size_t na, const void* b, size_t nb) {
+  if (ctx->sweep_base == dev_base && ctx->sweep_stream == st && ctx->sweep_tables.size() == na + nb &&
+      memcmp(ctx->sweep_tables.data(), a, na) == 0 && memcmp(ctx->sweep_tables.data() + na, b, nb) == 0)
+    return true;
+  ctx->sweep_tables.resize(na + nb);
+  memcpy(ctx->sweep_tables.data(), a, na);
+  memcpy(ctx->sweep_tables.data() + na, b, nb);
+  ctx->sweep_base = dev_base;
+  ctx->sweep_stream = st;
+  return false;
+}
 void* scratch(Ctx* ctx, size_t bytes) {
   if (bytes <= ctx->scratch_bytes) return ctx->scratch_buf;
   // the old buffer may still be in use by queued work on some stream
@@ -83,6 +98,7 @@ void* scratch(Ctx* ctx, size_t bytes) {
   if (cudaMalloc(&p, want) != cudaSuccess) { cudaGetLastError(); return nullptr; }
   ctx->scratch_buf = p;
   ctx->scratch_bytes = want;
+  ctx->sweep_base = nullptr;
   return p;
 }
 

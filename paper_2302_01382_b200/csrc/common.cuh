@@ -23,6 +23,9 @@ int sm_count(Ctx* ctx);
 int device_of(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);
+// true when the same two host tables were the last ones uploaded to this scratch address on
+// this context in this stream (the caller may then skip the upload); records them otherwise
+bool sweep_tables_cached(Ctx* ctx, const void* dev_base, cudaStream_t st, const void* a, size_t na, const void* b, size_t nb);
 // optional per-launch timing of one kernel class (0 = int8 GEMM, 1 = bf16 GEMM) with CUDA events
 void prof_begin(Ctx* ctx, int cls, cudaStream_t st);
 void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st);

@@ -22,6 +22,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kNB = 7;                       // bit widths 2..8
 constexpr float kMagic = 12582912.0f;        // 1.5 * 2^23
+constexpr int kRing = 3;                     // shared-memory row stages per thread
 constexpr int kItemFloatsMin = 8 * 1024;     // elements per work item (one block): bounds
 constexpr int kItemFloatsMax = 256 * 1024;
 
@@ -125,21 +126,14 @@ sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tenso
   const int n_iter = (int)((row1 - row0 + nteams - 1) / nteams);
   const float A_tensor = per_tensor ? tensor_absmax[d.tensor] : 0.0f;
 
-  __shared__ float smax[kThreads / 32];
+  __shared__ float smax2[2][kThreads / 32];
+  int row_parity = 0;
 
   double dacc[kNB];
 #pragma unroll
   for (int j = 0; j < kNB; ++j) dacc[j] = 0.0;
   float amax_blk = 0.0f;
 
-  auto load_row = [&](float4 (&dst)[V], int64_t row) {
-    const float4* p = reinterpret_cast<const float4*>(d.w + row * (int64_t)d.cols);
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-      int c = tl + v * T;
-      dst[v] = (row < row1 && c < c4) ? __ldg(p + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-  };
   auto process_row = [&](const float4 (&cur)[V]) {
     float m = 0.0f;
 #pragma unroll
@@ -148,12 +142,15 @@ sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tenso
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (T > 32) {
-      if (lane == 0) smax[threadIdx.x >> 5] = m;
-      __syncthreads();
+      // the team's warps exchange their maxima through shared memory; a named barrier per team
+      // keeps other teams running, and alternating slots make one barrier per row enough
+      float* slot = smax2[row_parity];
+      if (lane == 0) slot[threadIdx.x >> 5] = m;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(T) : "memory");
       const int w0 = team * (T >> 5);
-      m = smax[w0];
-      for (int w = 1; w < (T >> 5); ++w) m = fmaxf(m, smax[w0 + w]);
-      __syncthreads();
+      m = slot[w0];
+      for (int w = 1; w < (T >> 5); ++w) m = fmaxf(m, slot[w0 + w]);
+      row_parity ^= 1;
     }
     amax_blk = fmaxf(amax_blk, m);
     if (per_tensor) m = A_tensor;
@@ -181,17 +178,39 @@ sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tenso
     for (int j = 0; j < kNB; ++j) dacc[j] += (double)(facc[j].x + facc[j].y);
   };
 
-  // two register buffers, used alternately: the next row is in flight while this one is processed
-  float4 ra[V], rb[V];
-  load_row(ra, row0 + team);
-  for (int it = 0; it < n_iter; it += 2) {
-    load_row(rb, row0 + (int64_t)(it + 1) * nteams + team);   // zeros past the end
-    process_row(ra);
-    if (it + 1 < n_iter) {
-      load_row(ra, row0 + (int64_t)(it + 2) * nteams + team);
-      process_row(rb);
+  // Rows stream through a three-stage ring in shared memory filled by cp.async, two rows ahead
+  // of the one being processed: enough loads in flight to cover HBM latency without holding
+  // future rows in registers.  Every thread copies and reads back only its own 16-byte slots, so
+  // no barrier is needed between the copy and the read.
+  extern __shared__ float4 ring[];                       // [kRing][V][kThreads]
+  auto issue_row = [&](int stage, int64_t row) {
+    const float4* p = reinterpret_cast<const float4*>(d.w + row * (int64_t)d.cols);
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const int c = tl + v * T;
+      float4* dst = &ring[(stage * V + v) * kThreads + threadIdx.x];
+      if (row < row1 && c < c4) {
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(p + c) : "memory");
+      } else {
+        *dst = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  issue_row(0, row0 + team);
+  issue_row(1, row0 + (int64_t)nteams + team);
+  int stage = 0;
+  for (int it = 0; it < n_iter; ++it) {
+    int nxt = stage + 2; if (nxt >= kRing) nxt -= kRing;
+    issue_row(nxt, row0 + (int64_t)(it + 2) * nteams + team);      // zeros past the end
+    asm volatile("cp.async.wait_group 2;" ::: "memory");            // the row of this iteration has landed
+    float4 cur[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) cur[v] = ring[(stage * V + v) * kThreads + threadIdx.x];
+    process_row(cur);
+    if (++stage == kRing) stage = 0;
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   block_reduce_store(dacc, amax_blk, partial + (int64_t)blockIdx.x * 8);
 }
 
@@ -279,7 +298,13 @@ sweep_finalize_kernel(const double* __restrict__ partial, const TensorItems* __r
 template <int V>
 void launch_rows(const SweepDesc* d, int n, int items, int per_tensor, const float* amax, int jlo, int jhi,
                  double* partial, cudaStream_t st) {
-  sweep_rows_kernel<V><<<items, kThreads, 0, st>>>(d, n, per_tensor, amax, jlo, jhi, partial);
+  constexpr size_t smem = (size_t)kRing * V * kThreads * sizeof(float4);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(sweep_rows_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    attr_set = true;
+  }
+  sweep_rows_kernel<V><<<items, kThreads, smem, st>>>(d, n, per_tensor, amax, jlo, jhi, partial);
 }
 
 }  // namespace
@@ -349,9 +374,14 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
     group_desc0[c] = (int)flat.size();
     flat.insert(flat.end(), groups[c].begin(), groups[c].end());
   }
-  cudaError_t e = cudaMemcpyAsync(ddev, flat.data(), desc_bytes, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(tidev, titems.data(), ti_bytes, cudaMemcpyHostToDevice, st);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "sweep descriptor upload");
+  // the tables only depend on the tensor list: a repeated sweep of the same tensors (same scratch
+  // buffer) finds them on the device already
+  cudaError_t e = cudaSuccess;
+  if (!sweep_tables_cached(ctx, base, st, flat.data(), desc_bytes, titems.data(), ti_bytes)) {
+    e = cudaMemcpyAsync(ddev, flat.data(), desc_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(tidev, titems.data(), ti_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "sweep descriptor upload");
+  }
 
   if (per_tensor) {
     for (int t = 0; t < n_tensors; ++t) {
