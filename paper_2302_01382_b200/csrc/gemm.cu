@@ -198,35 +198,44 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 
 // Writes one warp's 32-row x 32-column piece of an output.  Each thread holds its row's 32
 // elements packed into WORDS 32-bit words (32: fp32 / int32, 16: bf16, 8: int8).
-// Staged path: the warp lays the piece out in its 4 KB shared-memory buffer (128-byte rows use
-// the 128B swizzle so the 16-byte writes spread over all banks) and one lane issues a TMA store,
-// which writes whole rows and clips at the matrix edge.  Direct path (outputs whose row pitch is
-// not a multiple of 16 bytes): per-thread stores.
+// Staged path: the warp lays the piece out in one of its two shared-memory slots and one lane
+// issues a TMA store, which writes whole rows and clips at the matrix edge.  Direct path
+// (outputs whose row pitch is not a multiple of 16 bytes): per-thread stores.
 template <int WORDS>
 __device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap* map, const uint32_t (&w)[WORDS],
                                             bool row_ok, int ncols, int64_t row, int row0, int col0,
                                             uint32_t stage, uint32_t stage_bytes, uint32_t& cursor, int lane) {
   constexpr int kRowBytes = WORDS * 4;
   constexpr int kElemBytes = kRowBytes / 32;
-  constexpr int kPieceBytes = 32 * kRowBytes;
   if (o.tma) {
-    // Pieces fill the warp's buffer one after the other; when the next one does not fit,
-    // wait until the TMA engine has read everything issued so far and start over.
-    if (cursor + kPieceBytes > stage_bytes) {
-      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-      __syncwarp();
-      cursor = 0;
-    }
-    const uint32_t base = stage + cursor;      // 1 KB-aligned: piece sizes are 1, 2 or 4 KB
-    cursor += kPieceBytes;
+    // The warp's buffer holds two slots used alternately: before a slot is rewritten only the
+    // store issued two pieces ago must have been read by the TMA engine (at most one store
+    // stays pending).  4-byte outputs go out as two 16-column pieces of 64-byte rows (64B
+    // swizzle: the 16-byte writes of eight lanes then cover all banks).
+    const uint32_t slot_bytes = stage_bytes >> 1;
+    constexpr int kHalves = (WORDS == 32) ? 2 : 1;
 #pragma unroll
-    for (int j = 0; j < WORDS / 4; ++j) {
-      const int jj = (WORDS == 32) ? (j ^ (lane & 7)) : j;
-      st_shared_v4(base + lane * kRowBytes + jj * 16, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+    for (int h = 0; h < kHalves; ++h) {
+      if (h == 1 && ncols <= 16) break;                 // warp-uniform: the second half lies outside
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      __syncwarp();
+      const uint32_t base = stage + (cursor & 1u) * slot_bytes;
+      ++cursor;
+      if (WORDS == 32) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int js = j ^ ((lane >> 1) & 3);
+          st_shared_v4(base + lane * 64 + js * 16, w[16 * h + 4 * j], w[16 * h + 4 * j + 1], w[16 * h + 4 * j + 2], w[16 * h + 4 * j + 3]);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < WORDS / 4; ++j)
+          st_shared_v4(base + lane * kRowBytes + j * 16, w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) tma_store_2d(map, base, col0 + 16 * h, row0);
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    if (lane == 0) tma_store_2d(map, base, col0, row0);
     return;
   }
   if (!row_ok) return;
@@ -506,7 +515,7 @@ int make_map(Ctx* ctx, CUtensorMap* map, const void* ptr, int is_bf16, int64_t k
   return QCFG_OK;
 }
 
-// Tensor map of an output matrix [m x n] for stores of 32 x 32-element pieces.  Returns false
+// Tensor map of an output matrix [m x n] for stores of 32-row pieces (32 columns, or 16 for 4-byte elements).  Returns false
 // (direct stores are used instead) when the pointer or the row pitch is not 16-byte aligned.
 bool make_out_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
   int esz; CUtensorMapDataType dt;
@@ -519,10 +528,10 @@ bool make_out_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
   if (((uintptr_t)o.ptr & 15) || ((o.ld * esz) & 15)) return false;
   cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)m};
   cuuint64_t strides[1] = {(cuuint64_t)(o.ld * esz)};
-  cuuint32_t box[2] = {32, 32};
+  cuuint32_t box[2] = {esz == 4 ? 16u : 32u, 32};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(map, dt, 2, o.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        esz == 4 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        esz == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
                         CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -585,7 +594,7 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   for (int i = 0; i < kNumOuts; ++i)
     if (p.outs[i].kind) p.outs[i].tma = make_out_map(&om.m[i], p.outs[i], g.m, g.n) ? 1 : 0;
 
-  // staging per epilogue warp: two 1 KB pieces when only int8 codes are written, else one 4 KB piece
+  // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
   bool wide = false;
   for (int i = 0; i < kNumOuts; ++i) if (p.outs[i].kind >= 2 && p.outs[i].tma) wide = true;
   p.epi_bytes = wide ? 4096 : 2048;
