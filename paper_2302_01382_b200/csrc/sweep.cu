@@ -109,7 +109,7 @@ __device__ __forceinline__ void err8(float2 x, float2 s, float2 inv, float2& acc
 // Rows of up to 32*V*team float4; cols % 4 == 0 and 16-byte aligned rows.  All 7 bit widths are
 // always evaluated (a narrower request only selects columns in the finalize kernel).
 template <int V>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 3)
 sweep_rows_kernel(const SweepDesc* __restrict__ descs, int n_desc, int per_tensor,
                   const float* __restrict__ tensor_absmax, int jlo, int jhi,
                   double* __restrict__ partial) {
