@@ -89,7 +89,8 @@ int qcfg_set_fusion(qcfg_ctx* ctx, int enabled);
 
 /* Per-launch timing of the GEMM kernel with CUDA events recorded on the launching stream
  * (off by default; a few microseconds of host time per launch when on).  kernel_class 0 is
- * the int8 GEMM, 1 the bf16 GEMM.  qcfg_profile_read waits for the recorded launches, then
+ * the int8 GEMM, 1 the bf16 GEMM, 2 every other kernel of the library (except the sweep's
+ * finalize step).  qcfg_profile_read waits for the recorded launches, then
  * returns the summed kernel time (ms), the number of launches and the summed algorithmic
  * operations (2*m*n*k per launch) since the last reset.  Outputs may be NULL.            */
 int qcfg_profile_enable(qcfg_ctx* ctx, int enabled);

@@ -29,8 +29,8 @@ struct Ctx {
   std::vector<cudaEvent_t> ev;      // pairs: ev[2i] before, ev[2i+1] after
   std::vector<int> ev_cls;
   size_t ev_used = 0;               // pairs in flight
-  double prof_ms[2] = {0, 0}, prof_ops[2] = {0, 0};
-  int64_t prof_n[2] = {0, 0};
+  double prof_ms[3] = {0, 0, 0}, prof_ops[3] = {0, 0, 0};
+  int64_t prof_n[3] = {0, 0, 0};
 };
 
 constexpr size_t kProfPairs = 8192;
@@ -452,7 +452,7 @@ int qcfg_profile_enable(qcfg_ctx* ctx, int enabled) {
   return QCFG_OK;
 }
 int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* launches, double* ops, int reset) {
-  if (!ctx || kernel_class < 0 || kernel_class > 1) return QCFG_EINVAL;
+  if (!ctx || kernel_class < 0 || kernel_class > 2) return QCFG_EINVAL;
   Ctx* c = &ctx->c;
   prof_drain(c);
   if (ms) *ms = c->prof_ms[kernel_class];

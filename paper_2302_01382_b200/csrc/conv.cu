@@ -46,7 +46,9 @@ int launch_maxpool3s2(Ctx* ctx, const float* src, int64_t B, int H, int W, int C
   const int vec = (C % 4 == 0 && (uintptr_t)src % 16 == 0 && (uintptr_t)dst % 16 == 0) ? 1 : 0;
   const int64_t total = B * OH * OW * (vec ? C / 4 : C);
   if (total == 0) return QCFG_OK;
+  prof_begin(ctx, 2, st);
   maxpool3s2_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(src, B, H, W, C, OH, OW, dst, vec);
+  prof_end(ctx, 2, 0.0, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "maxpool launch");
 }
@@ -68,7 +70,9 @@ __global__ void __launch_bounds__(256) avgpool_kernel(const float* __restrict__ 
 
 int launch_avgpool(Ctx* ctx, const float* src, int64_t B, int HW, int C, float* dst, cudaStream_t st) {
   if (B * C == 0) return QCFG_OK;
+  prof_begin(ctx, 2, st);
   avgpool_kernel<<<(unsigned)((B * C + 255) / 256), 256, 0, st>>>(src, B, HW, C, dst);
+  prof_end(ctx, 2, 0.0, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "avgpool launch");
 }
@@ -157,8 +161,10 @@ int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, 
   const int vec = (C % 8 == 0 && (uintptr_t)src % 16 == 0) ? 1 : 0;
   const int64_t total = rows * (ldq >> 3);
   const unsigned blocks = (unsigned)((total + 255) / 256);
+  prof_begin(ctx, 2, st);
   if (bits == 16) im2col_quantize_kernel<true><<<blocks, 256, 0, st>>>(src, rows, g, 1.0f, 0.0f, q, ldq, vec);
   else im2col_quantize_kernel<false><<<blocks, 256, 0, st>>>(src, rows, g, inv_scale, qmax_of(bits), q, ldq, vec);
+  prof_end(ctx, 2, 0.0, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "im2col launch");
 }

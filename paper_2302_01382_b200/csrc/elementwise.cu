@@ -97,12 +97,16 @@ int launch_absmax(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t 
     int64_t cap = (int64_t)sm_count(ctx) * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
+    prof_begin(ctx, 2, st);
     absmax_tensor_kernel<<<(unsigned)blocks, 256, 0, st>>>(x, rows, cols, ld, vec,
                                                             reinterpret_cast<unsigned*>(absmax));
+    prof_end(ctx, 2, 0.0, st);
   } else {
     if (rows == 0) return QCFG_OK;
     int64_t blocks = (rows + 7) / 8;
+    prof_begin(ctx, 2, st);
     absmax_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(x, rows, cols, ld, vec, absmax);
+    prof_end(ctx, 2, 0.0, st);
   }
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "absmax launch");
@@ -127,7 +131,9 @@ __global__ void scales_kernel(const float* __restrict__ absmax, int64_t n, float
 int launch_scales(Ctx* ctx, const float* absmax, int64_t n, int bits, float* scale, float* inv_scale,
                   cudaStream_t st) {
   if (n == 0) return QCFG_OK;
+  prof_begin(ctx, 2, st);
   scales_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(absmax, n, qmax_of(bits), scale, inv_scale);
+  prof_end(ctx, 2, 0.0, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "scales launch");
 }
@@ -193,10 +199,14 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
   const int64_t total = rows * (ldq >> 3);
   const unsigned blocks = (unsigned)((total + 255) / 256);
   if (bits == 16) {
+    prof_begin(ctx, 2, st);
     quantize_kernel<true><<<blocks, 256, 0, st>>>(x, rows, cols, ld, nullptr, 1.0f, 0, 0.0f, q, ldq, vec);
+    prof_end(ctx, 2, 0.0, st);
   } else {
+    prof_begin(ctx, 2, st);
     quantize_kernel<false><<<blocks, 256, 0, st>>>(x, rows, cols, ld, inv_scale_ptr, inv_scale_val,
                                                    granularity == QCFG_PER_ROW, qmax_of(bits), q, ldq, vec);
+    prof_end(ctx, 2, 0.0, st);
   }
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "quantize launch");

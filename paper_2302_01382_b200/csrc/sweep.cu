@@ -395,6 +395,7 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
     const SweepDesc* d = ddev + group_desc0[c];
     const int n = (int)groups[c].size();
     double* part = partial + (int64_t)group_item0[c] * 8;
+    prof_begin(ctx, 2, st);
     switch (c) {
       case 0: sweep_generic_kernel<<<group_items[c], kThreads, 0, st>>>(d, n, per_tensor, absmax, jlo, jhi, part); break;
       case 1: launch_rows<1>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
@@ -406,6 +407,7 @@ int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int
       case 7: launch_rows<7>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
       default: launch_rows<8>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
     }
+    prof_end(ctx, 2, 0.0, st);
     count_launch(ctx);
     e = cudaGetLastError();
     if (e != cudaSuccess) return check_cuda(ctx, e, "sweep launch");
@@ -537,6 +539,7 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
     const SweepDesc* d = S->descs + group_desc0[c];
     const int n = class_count[c];
     double* part = S->partial + (int64_t)group_item0[c] * 8;
+    prof_begin(ctx, 2, st);
     switch (c) {
       case 0: sweep_generic_kernel<<<group_items[c], kThreads, 0, st>>>(d, n, per_tensor, absmax, jlo, jhi, part); break;
       case 1: launch_rows<1>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
@@ -548,6 +551,7 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
       case 7: launch_rows<7>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
       default: launch_rows<8>(d, n, group_items[c], per_tensor, absmax, jlo, jhi, part, st); break;
     }
+    prof_end(ctx, 2, 0.0, st);
     count_launch(ctx);
     e = cudaGetLastError();
     if (e != cudaSuccess) return check_cuda(ctx, e, "static sweep launch");
