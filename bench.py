@@ -191,8 +191,15 @@ class Job:
         self.sse = torch.empty((len(self.weights), 7), dtype=torch.float64, device="cuda")
         self.amax = torch.empty(len(self.weights), dtype=torch.float32, device="cuda")
         self.sizes = np.array([a.size for a in w.weights], dtype=np.float64)
-        self.out = torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32, device="cuda")
-        self.ys = [None] * (len(w.layers) - 1) + [self.out]
+        # two result buffers used alternately, so that the device-to-host copy of one evaluation's
+        # result can overlap the next evaluation (end-to-end leg)
+        self.outs = [torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32, device="cuda") for _ in range(2)]
+        self.out = self.outs[0]
+        self.ys2 = [[None] * (len(w.layers) - 1) + [o] for o in self.outs]
+        self.ys = self.ys2[0]
+        self.copy_stream = torch.cuda.Stream()
+        self.done = [torch.cuda.Event() for _ in range(2)]
+        self.copied = [None, None]
         self.last_ranking = None
 
     def ranking_from_sweep(self):
@@ -202,16 +209,31 @@ class Job:
         return np.argsort(eqe, kind="stable")
 
     def step(self, x=None, host_out=None):
+        torch = self.torch
         ctx, w = self.ctx, self.w
         x = self.x if x is None else x
         ctx.quant_error_sweep(self.weights, self.q.PER_ROW, 2, 8, sse=self.sse, absmax=self.amax)
         rank = self.ranking_from_sweep()
         self.last_ranking = rank
         self.model.calibrate_model(x, w.m)
-        for bits in wl.greedy_sequence(rank, w.accept):
-            self.model.eval_config(bits, x, w.m, self.ys)
-            if host_out is not None:
-                host_out.copy_(self.out, non_blocking=True)
+        main = torch.cuda.current_stream()
+        for i, bits in enumerate(wl.greedy_sequence(rank, w.accept)):
+            if host_out is None:
+                self.model.eval_config(bits, x, w.m, self.ys)
+                continue
+            k = i & 1
+            if self.copied[k] is not None:
+                main.wait_event(self.copied[k])          # the copy that read this buffer has finished
+            self.model.eval_config(bits, x, w.m, self.ys2[k])
+            self.done[k].record(main)
+            with torch.cuda.stream(self.copy_stream):
+                self.copy_stream.wait_event(self.done[k])
+                host_out[k].copy_(self.outs[k], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(self.copy_stream)
+                self.copied[k] = ev
+        if host_out is not None:
+            main.wait_stream(self.copy_stream)
 
 
 def run_gpu(args):
@@ -290,7 +312,7 @@ def run_gpu(args):
     e2e = None
     if not args.no_e2e:
         host_x = torch.from_numpy(w.x).pin_memory()
-        host_out = torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32).pin_memory()
+        host_out = [torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32).pin_memory() for _ in range(2)]
         x_dev = torch.empty_like(job.x)
         e2e_steps = max(1, min(args.steps, 3))
         barrier()
@@ -303,7 +325,7 @@ def run_gpu(args):
         barrier()
         e2e_ms = max_over_ranks(t0.elapsed_time(t1), world)
         h2d = host_x.numel() * 4
-        d2h = N_EVALS * host_out.numel() * 4 + job.sse.numel() * 8 + job.amax.numel() * 4 + 4 * len(w.layers)
+        d2h = N_EVALS * host_out[0].numel() * 4 + job.sse.numel() * 8 + job.amax.numel() * 4 + 4 * len(w.layers)
         e2e = {"value": world * N_EVALS * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps}
 
