@@ -329,6 +329,18 @@ def run_gpu(args):
         e2e = {"value": world * N_EVALS * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps}
 
+    # ---------------- the greedy search driver itself (Algorithm 2 through qcfg_search: every
+    # evaluation is followed by the fidelity reduction and a synchronisation)
+    search = None
+    if not args.no_e2e:
+        rank_now = [int(v) for v in job.last_ranking]
+        t0 = time.perf_counter()
+        bits_s, vis_s, acc_s, n_s = job.model.search(q.SEARCH_GREEDY, rank_now, [8, 4], 0.9, job.x, w.m)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        search = {"algorithm": "greedy", "bs": [8, 4], "target_fidelity": 0.9, "evals": int(n_s), "ms": 1e3 * dt,
+                  "evals_per_s": n_s / dt, "layers_at_4_bit": int(sum(1 for b in bits_s if b == 4))}
+
     if rank == 0:
         int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])
         achieved = (g_ops / max(g_n, 1)) / (g_ms / max(g_n, 1) * 1e-3) / 1e12 if g_n else 0.0
@@ -350,6 +362,7 @@ def run_gpu(args):
                          "how": "CUDA events around every launch in a second pass over the same steps"},
             "sweep": {"gbs": sweep_gbs, "ms": sweep_ms, "bytes": sweep_bytes, "hbm_peak_gbs": peaks["hbm_gbs"],
                       "frac": sweep_gbs / peaks["hbm_gbs"], "peak_source": peaks["_source"]},
+            "search": search,
             "gemm_bf16": {"tflops": (b_ops / (b_ms * 1e-3) / 1e12) if b_ms else None, "launches": int(b_n)},
         }
         if not args.no_cpu_baseline and world == 1:

@@ -221,6 +221,25 @@ int qcfg_model_weight_absmax(qcfg_model* model, int32_t layer, float* absmax_hos
 int qcfg_eval_config(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits,
                      const float* x_dev, int64_t m, float* const* y_dev, void* stream);
 
+/* The paper's two configuration searches as host drivers over qcfg_eval_config.
+ * QCFG_SEARCH_BISECTION is Algorithm 1, QCFG_SEARCH_GREEDY Algorithm 2.  order[n_layers] lists
+ * the layers by ascending sensitivity (e.g. the E_QE ranking from qcfg_quant_error_sweep);
+ * bs[n_bs] are the available bit widths.  The working configuration starts at max(bs); the
+ * other widths are visited from high to low; the halving steps of Algorithm 1 use floor
+ * division and the prefix finally written is the largest one that met the target.
+ * "Accuracy" needs data and labels the library does not have; the drivers use the fidelity
+ * a = 1 - ||y - y_ref||_2 / ||y_ref||_2 of the LAST layer's fp32 output, y_ref being the output
+ * with every layer at max(bs), and accept a candidate when a >= target.
+ * Outputs (HOST): bits_out[n_layers] the final configuration; optionally visited
+ * [capacity x n_layers] the configurations evaluated, in order, and accuracies[capacity] their
+ * fidelities (the first `capacity` evaluations are recorded); n_evals the number of
+ * evaluations.  Synchronises the stream after every evaluation.                              */
+enum { QCFG_SEARCH_BISECTION = 0, QCFG_SEARCH_GREEDY = 1 };
+int qcfg_search(qcfg_ctx* ctx, qcfg_model* model, int algorithm, const int32_t* order,
+                const uint8_t* bs, int32_t n_bs, double target, const float* x_dev, int64_t m,
+                uint8_t* bits_out, uint8_t* visited, double* accuracies, int32_t capacity,
+                int32_t* n_evals, void* stream);
+
 /* Parity taps for layer `layer` of the LAST qcfg_eval_config call (same stream order):
  * the int8 codes of its GEMM input (qx_dev, [rows x k_in] dense, or NULL), of its weight
  * (qw_dev, [n_out x k_in] dense, or NULL) and its raw int32 accumulators (acc_dev,

@@ -17,6 +17,7 @@ from .build import LIB, build_library
 OK = 0
 PER_TENSOR, PER_ROW = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
+SEARCH_BISECTION, SEARCH_GREEDY = 0, 1
 STATUS_NAMES = ["OK", "EINVAL", "EBITS", "ESHAPE", "EALIGN", "ENOMEM", "ENONFINITE", "EARCH", "ECUDA",
                 "ETIMEOUT", "EUNIMPL", "ESTATE"]
 EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT, EUNIMPL, ESTATE = range(1, 12)
@@ -25,7 +26,7 @@ EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error",
            "qcfg_set_fusion", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
-           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_debug_dump"]
+           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_search", "qcfg_debug_dump"]
 
 
 class QcfgError(RuntimeError):
@@ -77,6 +78,8 @@ def load_library() -> C.CDLL:
         "qcfg_model_weight_absmax": [vp, i32, C.POINTER(f32)],
         "qcfg_eval_config": [vp, vp, C.POINTER(C.c_uint8), vp, i64, C.POINTER(vp), vp],
         "qcfg_debug_dump": [vp, vp, i32, vp, vp, vp, vp],
+        "qcfg_search": [vp, vp, ci, C.POINTER(i32), C.POINTER(C.c_uint8), i32, C.c_double, vp, i64, C.POINTER(C.c_uint8),
+                        C.POINTER(C.c_uint8), C.POINTER(C.c_double), i32, C.POINTER(i32), vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -285,6 +288,21 @@ class Model:
         if y is not None:
             yp = (C.c_void_p * n)(*[None if t is None else t.data_ptr() for t in y])
         self.ctx._check(self.ctx.lib.qcfg_eval_config(self.ctx.h, self.h, b, _ptr(x), m, yp, _stream(stream)))
+
+    def search(self, algorithm: int, order, bs, target: float, x: torch.Tensor, m: int, capacity: int = 4096, stream=None):
+        """Algorithm 1 (algorithm=0, bisection) or 2 (1, greedy).  Returns (bits, visited configurations, fidelities)."""
+        n = len(self.layers)
+        order_a = (C.c_int32 * n)(*[int(v) for v in order])
+        bs_a = (C.c_uint8 * len(bs))(*[int(v) for v in bs])
+        bits = (C.c_uint8 * n)()
+        visited = (C.c_uint8 * (capacity * n))()
+        acc = (C.c_double * capacity)()
+        n_evals = C.c_int32()
+        self.ctx._check(self.ctx.lib.qcfg_search(self.ctx.h, self.h, algorithm, order_a, bs_a, len(bs), float(target), _ptr(x), m,
+                                                 bits, visited, acc, capacity, C.byref(n_evals), _stream(stream)))
+        k = min(n_evals.value, capacity)
+        vis = [list(visited[i * n:(i + 1) * n]) for i in range(k)]
+        return list(bits), vis, list(acc[:k]), n_evals.value
 
     def debug_dump(self, layer: int, qx: Optional[torch.Tensor], qw: Optional[torch.Tensor], acc: Optional[torch.Tensor], stream=None):
         self.ctx._check(self.ctx.lib.qcfg_debug_dump(self.ctx.h, self.h, layer, _ptr(qx), _ptr(qw), _ptr(acc), _stream(stream)))

@@ -1,5 +1,6 @@
 // C-ABI of the library: context, model (layer table, weight-code cache, calibration tables)
 // and the host planner that turns one bit configuration into a sequence of kernel launches.
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -157,6 +158,7 @@ struct Model {
   bool calibrated = false;
   bool evaluated = false;
   DevBuf act_absmax_dev;           // fp32 [n_layers], filled by calibration
+  DevBuf search_ref, search_out, search_partial;   // buffers of the search drivers
   int64_t last_m = 0;
 };
 
@@ -637,6 +639,7 @@ int qcfg_model_destroy(qcfg_model* model) {
     for (auto& W : S.wc) { W.codes.release(); W.scale.release(); W.inv.release(); }
   }
   M->act_absmax_dev.release();
+  M->search_ref.release(); M->search_out.release(); M->search_partial.release();
   delete model;
   return QCFG_OK;
 }
@@ -695,6 +698,122 @@ int qcfg_eval_config(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, cons
   if (rc) return rc;
   M->evaluated = true;
   M->last_m = m;
+  return QCFG_OK;
+}
+
+// ---- search drivers (Algorithms 1 and 2 over qcfg_eval_config) ---------------------------------
+
+namespace {
+
+struct SearchState {
+  qcfg_ctx* ctx; qcfg_model* model;
+  const float* x; int64_t m; cudaStream_t st;
+  int n; int64_t out_elems; int blocks;
+  std::vector<float*> ys;
+  std::vector<double> host_partial;
+  uint8_t* visited; int32_t cap; double* acc_out; int32_t evals;
+  int rc;
+};
+
+// accuracy proxy of one configuration: 1 - ||y - ref||_2 / ||ref||_2 on the last layer's output
+double search_evaluate(SearchState& S, const std::vector<uint8_t>& cfg) {
+  Model* M = &S.model->m;
+  Ctx* c = &S.ctx->c;
+  if (S.rc) return 0.0;
+  S.rc = qcfg_eval_config(S.ctx, S.model, cfg.data(), S.x, S.m, S.ys.data(), S.st);
+  if (!S.rc) S.rc = launch_sqdiff(c, (const float*)M->search_out.p, (const float*)M->search_ref.p, S.out_elems,
+                                  (double*)M->search_partial.p, S.blocks, S.st);
+  if (!S.rc) S.rc = check_cuda(c, cudaMemcpyAsync(S.host_partial.data(), M->search_partial.p, (size_t)S.blocks * 16,
+                                                  cudaMemcpyDeviceToHost, S.st), "fidelity copy");
+  if (!S.rc) S.rc = qcfg_sync_status(S.ctx, S.st);
+  if (S.rc) return 0.0;
+  double d2 = 0.0, r2 = 0.0;
+  for (int b = 0; b < S.blocks; ++b) { d2 += S.host_partial[2 * b]; r2 += S.host_partial[2 * b + 1]; }
+  const double a = r2 > 0.0 ? 1.0 - std::sqrt(d2 / r2) : (d2 == 0.0 ? 1.0 : 0.0);
+  if (S.evals < S.cap) {
+    if (S.visited) memcpy(S.visited + (size_t)S.evals * S.n, cfg.data(), S.n);
+    if (S.acc_out) S.acc_out[S.evals] = a;
+  }
+  S.evals++;
+  return a;
+}
+
+}  // namespace
+
+int qcfg_search(qcfg_ctx* ctx, qcfg_model* model, int algorithm, const int32_t* order, const uint8_t* bs, int32_t n_bs,
+                double target, const float* x_dev, int64_t m, uint8_t* bits_out, uint8_t* visited, double* accuracies,
+                int32_t capacity, int32_t* n_evals, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  const int n = (int)M->L.size();
+  if (!order || !bs || n_bs < 1 || !x_dev || m <= 0 || !bits_out || capacity < 0)
+    return set_error(c, QCFG_EINVAL, "search: null pointer or bad size");
+  if (algorithm != QCFG_SEARCH_BISECTION && algorithm != QCFG_SEARCH_GREEDY) return set_error(c, QCFG_EINVAL, "search: unknown algorithm");
+  if (!M->calibrated) return set_error(c, QCFG_ESTATE, "search: model is not calibrated");
+  std::vector<char> seen(n, 0);
+  for (int i = 0; i < n; ++i) {
+    if (order[i] < 0 || order[i] >= n || seen[order[i]]) return set_error(c, QCFG_EINVAL, "search: order is not a permutation of the layers");
+    seen[order[i]] = 1;
+  }
+  int top = 0;
+  for (int i = 0; i < n_bs; ++i) { if (!bits_ok(bs[i])) return set_error(c, QCFG_EBITS, "search: bit width %d", (int)bs[i]); if (bs[i] > top) top = bs[i]; }
+  std::vector<int> lower;                       // the other bit widths, high to low
+  for (int i = 0; i < n_bs; ++i) if (bs[i] != top) lower.push_back(bs[i]);
+  std::sort(lower.begin(), lower.end(), [](int a, int b) { return a > b; });
+  lower.erase(std::unique(lower.begin(), lower.end()), lower.end());
+
+  SearchState S{};
+  S.ctx = ctx; S.model = model; S.x = x_dev; S.m = m; S.st = (cudaStream_t)stream; S.n = n;
+  S.visited = visited; S.cap = capacity; S.acc_out = accuracies; S.evals = 0; S.rc = 0;
+  S.out_elems = layer_rows(M, n - 1, m) * M->L[n - 1].d.n_out;
+  S.blocks = c->sms * 4;
+  S.host_partial.resize((size_t)S.blocks * 2);
+  int rc = M->search_ref.ensure(c, (size_t)S.out_elems * 4);
+  if (!rc) rc = M->search_out.ensure(c, (size_t)S.out_elems * 4);
+  if (!rc) rc = M->search_partial.ensure(c, (size_t)S.blocks * 16);
+  if (rc) return rc;
+  S.ys.assign(n, nullptr);
+
+  // reference output: every layer at max(bs), the configuration both searches start from
+  std::vector<uint8_t> w(n, (uint8_t)top);
+  S.ys[n - 1] = (float*)M->search_ref.p;
+  rc = qcfg_eval_config(ctx, model, w.data(), x_dev, m, S.ys.data(), stream);
+  if (rc) return rc;
+  S.ys[n - 1] = (float*)M->search_out.p;
+
+  std::vector<int> ll(order, order + n);
+  if (algorithm == QCFG_SEARCH_BISECTION) {
+    for (int b : lower) {
+      int thr = (int)ll.size() / 2, upl = (int)ll.size(), lowl = 0;
+      for (;;) {
+        std::vector<uint8_t> lw(w);
+        for (int i = 0; i < thr; ++i) lw[ll[i]] = (uint8_t)b;
+        const double a = search_evaluate(S, lw);
+        if (S.rc) return S.rc;
+        const int old = thr;
+        if (a >= target) { lowl = thr; thr = thr + (upl - thr) / 2; }
+        else { upl = thr; thr = thr - (thr - lowl) / 2; }
+        if (thr == old) break;
+      }
+      for (int i = 0; i < lowl; ++i) w[ll[i]] = (uint8_t)b;
+      ll.resize(lowl);
+    }
+  } else {
+    for (int b : lower) {
+      std::vector<int> ql;
+      for (int l : ll) {
+        const uint8_t last = w[l];
+        w[l] = (uint8_t)b;
+        const double a = search_evaluate(S, w);
+        if (S.rc) return S.rc;
+        if (a >= target) ql.push_back(l); else w[l] = last;
+      }
+      ll.swap(ql);
+    }
+  }
+  memcpy(bits_out, w.data(), n);
+  if (n_evals) *n_evals = S.evals;
   return QCFG_OK;
 }
 

@@ -40,6 +40,8 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
                     const float* inv_scale_ptr, float inv_scale_val, int granularity, int bits,
                     void* q, int64_t ldq, cudaStream_t st);
 
+int launch_sqdiff(Ctx* ctx, const float* y, const float* ref, int64_t n, double* partial, int blocks, cudaStream_t st);
+
 // ----- conv.cu ------------------------------------------------------------------------
 int launch_maxpool3s2(Ctx* ctx, const float* src, int64_t B, int H, int W, int C, float* dst, cudaStream_t st);
 int launch_avgpool(Ctx* ctx, const float* src, int64_t B, int HW, int C, float* dst, cudaStream_t st);

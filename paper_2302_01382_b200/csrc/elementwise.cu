@@ -212,4 +212,36 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
   return check_cuda(ctx, cudaGetLastError(), "quantize launch");
 }
 
+
+// ------------------------------------------------------------------------------- output fidelity
+
+// Per-block partial sums of (y - ref)^2 and ref^2 in fp64 (fixed grid, fixed order: deterministic).
+__global__ void __launch_bounds__(256) sqdiff_kernel(const float* __restrict__ y, const float* __restrict__ ref,
+                                                     int64_t n, double* __restrict__ partial) {
+  double d2 = 0.0, r2 = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const double r = (double)__ldg(ref + i), d = (double)__ldg(y + i) - r;
+    d2 += d * d;
+    r2 += r * r;
+  }
+  d2 = warp_sum(d2);
+  r2 = warp_sum(r2);
+  __shared__ double sm[8][2];
+  if ((threadIdx.x & 31) == 0) { sm[threadIdx.x >> 5][0] = d2; sm[threadIdx.x >> 5][1] = r2; }
+  __syncthreads();
+  if (threadIdx.x < 2) {
+    double v = 0.0;
+    for (int w = 0; w < 8; ++w) v += sm[w][threadIdx.x];
+    partial[2 * blockIdx.x + threadIdx.x] = v;
+  }
+}
+
+int launch_sqdiff(Ctx* ctx, const float* y, const float* ref, int64_t n, double* partial, int blocks, cudaStream_t st) {
+  prof_begin(ctx, 2, st);
+  sqdiff_kernel<<<blocks, 256, 0, st>>>(y, ref, n, partial);
+  prof_end(ctx, 2, 0.0, st);
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "fidelity launch");
+}
+
 }  // namespace qcfg
