@@ -28,17 +28,23 @@ def main():
     ap.add_argument("--bits", type=int, default=8)
     ap.add_argument("--sweep", type=int, default=0, help="number of sweep calls to run after the evaluations")
     ap.add_argument("--seed", type=int, default=2)
+    ap.add_argument("--resnet", type=int, default=0, help="batch size: run the ResNet-50 table instead of a BERT stack")
+    ap.add_argument("--mixed", action="store_true", help="use the workload's drawn bit configuration instead of --bits")
     args = ap.parse_args()
 
-    w = wl.bert_stack(args.seed, args.tokens, args.hidden, args.ffn, args.blocks, bit_choices=None)
+    if args.resnet:
+        w = wl.resnet50(batch=args.resnet)
+    else:
+        w = wl.bert_stack(args.seed, args.tokens, args.hidden, args.ffn, args.blocks,
+                          bit_choices=(4, 8, 16) if args.mixed else None)
     ctx = Context(0)
     weights = [torch.from_numpy(a).cuda() for a in w.weights]
     x = torch.from_numpy(w.x).cuda()
     model = Model(ctx, w.layers, weights)
     model.calibrate_model(x, w.m)
-    out = torch.empty((w.m, w.layers[-1].n_out), device="cuda")
+    out = torch.empty((wl.layer_rows(w.layers, len(w.layers) - 1, w.m), w.layers[-1].n_out), device="cuda")
     ys = [None] * (len(w.layers) - 1) + [out]
-    bits = [args.bits] * len(w.layers)
+    bits = list(w.bits) if (args.mixed or args.resnet) and w.bits is not None else [args.bits] * len(w.layers)
     model.eval_config(bits, x, w.m, ys)          # builds the weight-code cache
     ctx.check_sync()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -50,7 +56,7 @@ def main():
     t_host = time.perf_counter() - t0
     ctx.check_sync()
     print(f"evaluations: host enqueue {1e3 * t_host / args.evals:.3f} ms, device {e0.elapsed_time(e1) / args.evals:.3f} ms each "
-          f"({len(w.layers)} layers, {args.tokens} tokens, {args.bits} bit)")
+          f"({len(w.layers)} layers, m = {w.m}, bits {sorted(set(int(b) for b in bits))})")
     if args.sweep:
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         sse, amax = ctx.quant_error_sweep(weights, PER_ROW)
