@@ -86,6 +86,10 @@ int64_t qcfg_launch_count(qcfg_ctx* ctx);
  * (default on).  Off: every layer's fp32 output is written and re-read by a separate quantize
  * kernel; results are bit-identical either way.                                           */
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled);
+/* Switches the two-CTA GEMM tiles (256 rows per CTA pair, cta_group::2; default on, used for
+ * outputs wider than 128 columns and more than 128 rows).  Off: every tile is 128 rows on one
+ * CTA.  Results are bit-identical either way.                                               */
+int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled);
 
 /* Per-launch timing of the GEMM kernel with CUDA events recorded on the launching stream
  * (off by default; a few microseconds of host time per launch when on).  kernel_class 0 is

@@ -20,6 +20,8 @@ struct Ctx {
   size_t scratch_bytes = 0;
   int64_t launches = 0;
   int fuse = 1;
+  int pair = 1;                     // two-CTA GEMM tiles where they apply
+  int pair_clusters[2] = {0, 0};
   char msg[512] = {0};
   // last sweep tables uploaded to the scratch buffer
   const void* sweep_base = nullptr;
@@ -64,6 +66,8 @@ void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st) {
 void count_launch(Ctx* ctx, int n) { ctx->launches += n; }
 unsigned* err_word(Ctx* ctx) { return ctx->err_dev; }
 int sm_count(Ctx* ctx) { return ctx->sms; }
+bool ctx_pair_enabled(Ctx* ctx) { return ctx->pair != 0; }
+int* pair_cluster_cache(Ctx* ctx) { return ctx->pair_clusters; }
 int device_of(Ctx* ctx) { return ctx->device; }
 
 int set_error(Ctx* ctx, int code, const char* fmt, ...) {
@@ -461,6 +465,11 @@ int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* laun
   if (launches) *launches = c->prof_n[kernel_class];
   if (ops) *ops = c->prof_ops[kernel_class];
   if (reset) { c->prof_ms[kernel_class] = 0; c->prof_n[kernel_class] = 0; c->prof_ops[kernel_class] = 0; }
+  return QCFG_OK;
+}
+int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled) {
+  if (!ctx) return QCFG_EINVAL;
+  ctx->c.pair = enabled ? 1 : 0;
   return QCFG_OK;
 }
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled) {

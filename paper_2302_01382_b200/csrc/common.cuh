@@ -20,6 +20,8 @@ int set_error(Ctx* ctx, int code, const char* fmt, ...);
 int check_cuda(Ctx* ctx, cudaError_t e, const char* what);
 unsigned* err_word(Ctx* ctx);
 int sm_count(Ctx* ctx);
+bool ctx_pair_enabled(Ctx* ctx);
+int* pair_cluster_cache(Ctx* ctx);   // [2]: resident CTA pairs of the int8 / bf16 pair kernels, 0 = not yet queried
 int device_of(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);

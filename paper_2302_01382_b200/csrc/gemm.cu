@@ -112,11 +112,52 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 
+// Pair flavour (two CTAs of a cluster work on one 256-row tile, cta_group::2): the load of either
+// CTA reports its bytes to the barrier of the pair's first CTA; shared-memory addresses of the
+// two CTAs differ in bit 24 of the shared::cluster window.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t x, int32_t y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar & kPeerBitMask), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {   // arrive on the first CTA's copy of the barrier
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerBitMask) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {       // arrives on this barrier in both CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <bool BF16>
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  if (BF16) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+  }
 }
 
 template <bool BF16>
@@ -331,7 +372,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
 
 // ---------------------------------------------------------------------------- the kernel
 
-template <bool BF16>
+template <bool BF16, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ OutMaps omaps, const __grid_constant__ GemmParams p) {
@@ -346,36 +387,61 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const uint32_t stage_bytes = (uint32_t)(BM + p.bn) * kStageKBytes;
+  // Pair flavour: the two CTAs of a cluster share one 256-row tile.  Each loads its own 128 rows
+  // of A and its own half of the tile's B rows; the first CTA issues the MMAs for both
+  // (cta_group::2), each CTA's TMEM receives the accumulators of its 128 rows.  p.tiles_m then
+  // counts 256-row tiles.
+  const int rank = PAIR ? (int)cluster_ctarank() : 0;
+  const int b_rows = PAIR ? (p.bn >> 1) : p.bn;                  // B rows held per stage by this CTA
+  const uint32_t stage_bytes = (uint32_t)(BM + b_rows) * kStageKBytes;
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
   const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16;
   const int num_tiles = p.tiles_m * p.tiles_n;
+  const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // first tile of this CTA (pair)
+  const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int rows_per_tile = PAIR ? 2 * BM : BM;
 
   // producer state (thread 0 only): next k-block to load
-  int ld_tile = blockIdx.x, ld_kb = 0, ld_s = 0;
+  int ld_tile = tile0, ld_kb = 0, ld_s = 0;
   uint32_t ld_ph = 0;
   const int k_elems = BF16 ? kStageKBytes / 2 : kStageKBytes;
   auto issue_load = [&]() {   // the stage's empty barrier must already have been passed
     const int tm = ld_tile % p.tiles_m, tn = ld_tile / p.tiles_m;
     const uint32_t a_dst = smem_u32(stage_base + (size_t)ld_s * stage_bytes);
-    mbar_expect_tx(full0 + 8 * ld_s, stage_bytes);
-    tma_load_2d(a_dst, &map_a, full0 + 8 * ld_s, ld_kb * k_elems, tm * BM);
-    tma_load_2d(a_dst + BM * kStageKBytes, &map_b, full0 + 8 * ld_s, ld_kb * k_elems, tn * p.bn);
+    if (PAIR) {
+      // the first CTA's barrier collects the bytes of both CTAs' loads
+      if (rank == 0) mbar_expect_tx(full0 + 8 * ld_s, 2 * stage_bytes);
+      tma_load_2d_pair(a_dst, &map_a, full0 + 8 * ld_s, ld_kb * k_elems, tm * rows_per_tile + rank * BM);
+      tma_load_2d_pair(a_dst + BM * kStageKBytes, &map_b, full0 + 8 * ld_s, ld_kb * k_elems, tn * p.bn + rank * b_rows);
+    } else {
+      mbar_expect_tx(full0 + 8 * ld_s, stage_bytes);
+      tma_load_2d(a_dst, &map_a, full0 + 8 * ld_s, ld_kb * k_elems, tm * BM);
+      tma_load_2d(a_dst + BM * kStageKBytes, &map_b, full0 + 8 * ld_s, ld_kb * k_elems, tn * p.bn);
+    }
     if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; }
-    if (++ld_kb == p.k_blocks) { ld_kb = 0; ld_tile += gridDim.x; }
+    if (++ld_kb == p.k_blocks) { ld_kb = 0; ld_tile += tile_step; }
   };
 
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, kEpiWarps); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {   // the same warp of both CTAs allocates for the pair
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+  }
+  if (PAIR) {     // both CTAs' barriers exist before either one's loads or arrivals can reach them
+    __syncthreads();
+    cluster_sync_all();
   }
   // Everything above touches no global memory, so under programmatic dependent launch it
   // overlaps the tail of the previous kernel in the stream; from here on its results are needed.
@@ -398,6 +464,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (!mbar_wait(empty0 + 8 * ld_s, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
         issue_load();
       }
+      if (PAIR && ok) {
+        // the peer's MMA completions still arrive on this CTA's stage barriers: drain them all
+        // before this CTA may exit (a stage never filled passes at once)
+        for (int i = 0; i < p.stages && ok; ++i) {
+          if (!mbar_wait(empty0 + 8 * ld_s, ld_ph ^ 1, abort_flag, p.err)) ok = false;
+          if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; }
+        }
+      }
       if (!ok) {
         // give copies already in flight a bounded time to land before the CTA exits
         const uint64_t t0 = global_timer();
@@ -406,11 +480,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       int t = 0;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+      for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
         const int a = t & 1;
         if (!mbar_wait(tempty0 + 8 * a, ((t >> 1) & 1) ^ 1, abort_flag, p.err)) { ok = false; break; }
         tc_fence_after();
@@ -423,12 +497,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
           for (int k4 = 0; k4 < kStageKBytes / kUmmaKBytes; ++k4) {
             // advancing the start address by 32 bytes (2 units) steps along K inside the swizzle atom
-            tc_mma<BF16>(d_tmem, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), p.idesc, (kb | k4) != 0);
+            if (PAIR) tc_mma_pair<BF16>(d_tmem, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), p.idesc, (kb | k4) != 0);
+            else tc_mma<BF16>(d_tmem, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), p.idesc, (kb | k4) != 0);
           }
-          tc_commit(empty0 + 8 * s);          // stage reusable once these MMAs have read it
+          if (PAIR) tc_commit_pair(empty0 + 8 * s); else tc_commit(empty0 + 8 * s);   // stage reusable once these MMAs have read it
           if (++s == p.stages) { s = 0; ph ^= 1; }
         }
-        if (ok) tc_commit(tfull0 + 8 * a);    // accumulator complete
+        if (ok) { if (PAIR) tc_commit_pair(tfull0 + 8 * a); else tc_commit(tfull0 + 8 * a); }   // accumulator complete
       }
     }
   } else {
@@ -444,10 +519,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     uint32_t cursor = 0;
     bool ok = true;
     int t = 0;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+    for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
       const int a = t & 1;
       const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-      const int row0 = tm * BM + quad * 32;
+      const int row0 = tm * rows_per_tile + rank * BM + quad * 32;
       const int col_base = tn * p.bn + c_begin * 32;
       // column scales of this warp's chunks, one column per lane and chunk, fetched while the
       // tensor cores are still working on the tile
@@ -473,13 +548,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (c == nch - 1) {   // the accumulator buffer is free again once this warp's columns sit in registers
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(tempty0 + 8 * a);
+          if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
         }
         epilogue_chunk<BF16>(p, omaps, v, c ? cs[1] : cs[0], row, row0, col_base + 32 * c, stage, cursor, lane);
       }
       if (nch == 0) {
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty0 + 8 * a);
+        if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
       }
     }
     // all TMA stores of this warp must have completed before the CTA's shared memory goes away
@@ -488,9 +563,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();     // the peer no longer signals this CTA's barriers nor uses its TMEM
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -547,8 +624,10 @@ int gemm_init(Ctx* ctx) {
       return set_error(ctx, QCFG_ECUDA, "cuTensorMapEncodeTiled entry point not found");
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  cudaError_t e = cudaFuncSetAttribute(gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   return check_cuda(ctx, e, "gemm smem attribute");
 }
 
@@ -567,13 +646,17 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   int bn = 256;
   if (g.n <= 32) bn = 32; else if (g.n <= 64) bn = 64; else if (g.n <= 128) bn = 128;
   p.bn = bn;
-  p.tiles_m = (int32_t)((g.m + BM - 1) / BM);
+  // pair flavour (two CTAs per 256-row tile, cta_group::2) for wide outputs with at least two
+  // row tiles: it halves the B bytes each SM pulls from L2, which is what limits the main loop
+  const bool pair = ctx_pair_enabled(ctx) && bn == 256 && g.m > BM && sm_count(ctx) >= 2;
+  const int tile_rows = pair ? 2 * BM : BM;
+  p.tiles_m = (int32_t)((g.m + tile_rows - 1) / tile_rows);
   p.tiles_n = (int32_t)((g.n + bn - 1) / bn);
-  const int stage_bytes = (BM + bn) * kStageKBytes;
+  const int stage_bytes = (BM + (pair ? bn / 2 : bn)) * kStageKBytes;
   p.is_bf16 = g.is_bf16;
   // instruction descriptor: D format (F32 = 1, S32 = 2) at bit 4, A/B format (BF16 = 1, S8 = 1)
   // at bits 7 and 10, both operands K-major, N/8 at bit 17, M/16 at bit 24
-  p.idesc = ((g.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+  p.idesc = ((g.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(tile_rows >> 4) << 24);
   p.scale_x = g.scale_x; p.scale_w = g.scale_w; p.act = g.act;
   p.residual = g.residual; p.ldr = g.ldr;
   if (g.acc && !g.is_bf16) { p.outs[0].kind = 4; p.outs[0].ptr = g.acc; p.outs[0].ld = g.n; }
@@ -604,12 +687,32 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
 
   CUtensorMap ma, mb;
   int rc = make_map(ctx, &ma, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
-  if (rc == QCFG_OK) rc = make_map(ctx, &mb, g.b, g.is_bf16, g.k, g.n, g.ldb, bn);
+  if (rc == QCFG_OK) rc = make_map(ctx, &mb, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
   if (rc != QCFG_OK) return rc;
 
   const int num_tiles = p.tiles_m * p.tiles_n;
   int grid = sm_count(ctx);
-  if (grid > num_tiles) grid = num_tiles;
+  if (pair) {
+    int* cached = pair_cluster_cache(ctx) + (g.is_bf16 ? 1 : 0);
+    if (*cached == 0) {     // how many CTA pairs the device keeps resident at once
+      cudaLaunchConfig_t q = {};
+      q.gridDim = dim3((unsigned)(grid & ~1));
+      q.blockDim = dim3(kGemmThreads);
+      q.dynamicSmemBytes = kSmemMax;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+      q.attrs = qa; q.numAttrs = 1;
+      int n = 0;
+      cudaError_t oe = g.is_bf16 ? cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true, true>, &q)
+                                 : cudaOccupancyMaxActiveClusters(&n, gemm_kernel<false, true>, &q);
+      if (oe != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = grid / 2; }
+      if (n > grid / 2) n = grid / 2;
+      *cached = n;
+    }
+    grid = 2 * (*cached);
+    if (grid > 2 * num_tiles) grid = 2 * num_tiles;
+  } else if (grid > num_tiles) grid = num_tiles;
   const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)kEpiWarps * p.epi_bytes + (size_t)stages * stage_bytes;
   // Programmatic dependent launch: the kernel's prologue (barrier set-up, TMEM allocation) may
   // start while the previous kernel in the stream drains; it waits (griddepcontrol.wait) before
@@ -619,14 +722,19 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pair ? 2 : 1;
   prof_begin(ctx, g.is_bf16 ? 1 : 0, st);
-  cudaError_t le = g.is_bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true>, ma, mb, om, p)
-                             : cudaLaunchKernelEx(&cfg, gemm_kernel<false>, ma, mb, om, p);
+  cudaError_t le;
+  if (pair) le = g.is_bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, true>, ma, mb, om, p)
+                           : cudaLaunchKernelEx(&cfg, gemm_kernel<false, true>, ma, mb, om, p);
+  else le = g.is_bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, false>, ma, mb, om, p)
+                      : cudaLaunchKernelEx(&cfg, gemm_kernel<false, false>, ma, mb, om, p);
   prof_end(ctx, g.is_bf16 ? 1 : 0, 2.0 * (double)g.m * (double)g.n * (double)g.k, st);
   if (le != cudaSuccess) return check_cuda(ctx, le, "gemm launch");
   count_launch(ctx);

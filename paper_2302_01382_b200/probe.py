@@ -30,6 +30,7 @@ def main():
     ap.add_argument("--seed", type=int, default=2)
     ap.add_argument("--resnet", type=int, default=0, help="batch size: run the ResNet-50 table instead of a BERT stack")
     ap.add_argument("--mixed", action="store_true", help="use the workload's drawn bit configuration instead of --bits")
+    ap.add_argument("--single-cta", action="store_true", help="128-row GEMM tiles on one CTA each instead of CTA pairs")
     args = ap.parse_args()
 
     if args.resnet:
@@ -38,6 +39,7 @@ def main():
         w = wl.bert_stack(args.seed, args.tokens, args.hidden, args.ffn, args.blocks,
                           bit_choices=(4, 8, 16) if args.mixed else None)
     ctx = Context(0)
+    ctx.set_pair_tiles(not args.single_cta)
     weights = [torch.from_numpy(a).cuda() for a in w.weights]
     x = torch.from_numpy(w.x).cuda()
     model = Model(ctx, w.layers, weights)

@@ -178,6 +178,30 @@ def test_gemm_i8_accumulators_and_rescale_bit_exact(ctx, m, n, k):
     np.testing.assert_array_equal(host(y).view(np.uint32), orc.dequant_output(ref, sx, sw).view(np.uint32))
 
 
+@pytest.mark.parametrize("m,n,k", [(5000, 1024, 272), (257, 300, 1040), (129, 2304, 64)])
+def test_gemm_pair_and_single_cta_tiles_agree(ctx, m, n, k):
+    """Outputs wider than 128 columns run on CTA pairs (256-row tiles); the single-CTA path must
+    give the same bits, also when a pair works through several tiles and when the second CTA's
+    rows or columns lie partly or wholly outside the matrix."""
+    import paper_2302_01382_b200 as q
+    rng = np.random.default_rng(m * 7 + n)
+    ld = (k + 15) // 16 * 16
+    qx, qw = _codes(rng, m, k, ld), _codes(rng, n, k, ld)
+    sw = (10.0 ** rng.uniform(-4, -2, n)).astype(np.float32)
+    res = []
+    for pair in (True, False):
+        ctx.set_pair_tiles(pair)
+        try:
+            y, acc = ctx.gemm_i8(dev(qx), dev(qw), k, 0.021, dev(sw), q.ACT_GELU_TANH, want_y=True, want_acc=True)
+            ctx.check_sync()
+        finally:
+            ctx.set_pair_tiles(True)
+        res.append((y, acc))
+    np.testing.assert_array_equal(host(res[0][1]), orc.int_gemm(qx[:, :k], qw[:, :k]))
+    assert torch.equal(res[0][1], res[1][1])
+    assert torch.equal(res[0][0].view(torch.int32), res[1][0].view(torch.int32))
+
+
 def test_gemm_i8_worst_case_magnitude(ctx):
     k = 4608
     qx = np.full((128, k), 127, np.int8)
