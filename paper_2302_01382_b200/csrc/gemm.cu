@@ -188,17 +188,11 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&v)[32
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128B swizzle, groups of 8
-// rows 1024 bytes apart (the layout a 128B-swizzled TMA box produces).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFF);          // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                         // descriptor version for sm_100
-  d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
-  return d;
-}
+// Shared-memory matrix descriptors used by the MMA issuer: K-major tile of 128-byte rows, 128B
+// swizzle, groups of 8 rows 1024 bytes apart (the layout a 128B-swizzled TMA box produces).
+// Bits 0-13 start address in 16-byte units, bit 16 leading byte offset (unused for swizzled
+// K-major), bits 32-45 stride byte offset between 8-row groups (1024 >> 4), bit 46 descriptor
+// version of sm_100, bits 61-63 layout type 2 = SWIZZLE_128B.
 
 // ---------------------------------------------------------------------------- epilogue math
 
@@ -402,24 +396,36 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int rows_per_tile = PAIR ? 2 * BM : BM;
 
   // producer state (thread 0 only): next k-block to load
+  // The producer and the MMA issuer share their scheduler with four epilogue warps that almost
+  // always have an instruction ready, so every instruction these two threads need per k-block
+  // costs them many cycles of waiting for an issue slot: their loops keep all addresses and
+  // coordinates in registers and update them incrementally.
   int ld_tile = tile0, ld_kb = 0, ld_s = 0;
   uint32_t ld_ph = 0;
   const int k_elems = BF16 ? kStageKBytes / 2 : kStageKBytes;
-  auto issue_load = [&]() {   // the stage's empty barrier must already have been passed
+  const uint32_t stage0 = smem_u32(stage_base);
+  uint32_t ld_dst = stage0, ld_bar = full0;      // stage address and its full barrier
+  int ld_x = 0, ld_ya = 0, ld_yb = 0;            // TMA coordinates of the next k-block
+  auto set_tile_coords = [&]() {
     const int tm = ld_tile % p.tiles_m, tn = ld_tile / p.tiles_m;
-    const uint32_t a_dst = smem_u32(stage_base + (size_t)ld_s * stage_bytes);
+    ld_ya = tm * rows_per_tile + rank * BM;
+    ld_yb = tn * p.bn + rank * b_rows;
+  };
+  set_tile_coords();
+  auto issue_load = [&]() {   // the stage's empty barrier must already have been passed
     if (PAIR) {
       // the first CTA's barrier collects the bytes of both CTAs' loads
-      if (rank == 0) mbar_expect_tx(full0 + 8 * ld_s, 2 * stage_bytes);
-      tma_load_2d_pair(a_dst, &map_a, full0 + 8 * ld_s, ld_kb * k_elems, tm * rows_per_tile + rank * BM);
-      tma_load_2d_pair(a_dst + BM * kStageKBytes, &map_b, full0 + 8 * ld_s, ld_kb * k_elems, tn * p.bn + rank * b_rows);
+      if (rank == 0) mbar_expect_tx(ld_bar, 2 * stage_bytes);
+      tma_load_2d_pair(ld_dst, &map_a, ld_bar, ld_x, ld_ya);
+      tma_load_2d_pair(ld_dst + BM * kStageKBytes, &map_b, ld_bar, ld_x, ld_yb);
     } else {
-      mbar_expect_tx(full0 + 8 * ld_s, stage_bytes);
-      tma_load_2d(a_dst, &map_a, full0 + 8 * ld_s, ld_kb * k_elems, tm * BM);
-      tma_load_2d(a_dst + BM * kStageKBytes, &map_b, full0 + 8 * ld_s, ld_kb * k_elems, tn * p.bn);
+      mbar_expect_tx(ld_bar, stage_bytes);
+      tma_load_2d(ld_dst, &map_a, ld_bar, ld_x, ld_ya);
+      tma_load_2d(ld_dst + BM * kStageKBytes, &map_b, ld_bar, ld_x, ld_yb);
     }
-    if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; }
-    if (++ld_kb == p.k_blocks) { ld_kb = 0; ld_tile += tile_step; }
+    ld_dst += stage_bytes; ld_bar += 8; ld_x += k_elems;
+    if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; ld_dst = stage0; ld_bar = full0; }
+    if (++ld_kb == p.k_blocks) { ld_kb = 0; ld_x = 0; ld_tile += tile_step; set_tile_coords(); }
   };
 
   if (threadIdx.x == 0) {
@@ -461,7 +467,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (lane == 0) {
       bool ok = true;
       while (ld_tile < num_tiles) {
-        if (!mbar_wait(empty0 + 8 * ld_s, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
+        if (!mbar_wait(ld_bar + 8 * kMaxStages, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
         issue_load();
       }
       if (PAIR && ok) {
@@ -481,27 +487,40 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
+      // Descriptor low words (start address field, 16-byte units) of the four K steps of the
+      // current stage's A and B tiles; the high word is the same for all.
+      constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t lo0 = ((stage0 >> 4) & 0x3FFFu) | (1u << 16);
+      const uint32_t lo_step = stage_bytes >> 4;
+      constexpr uint32_t kBOff = (uint32_t)(BM * kStageKBytes) >> 4;
+      uint32_t lo = lo0, fb = full0;
       int s = 0; uint32_t ph = 0;
       bool ok = true;
       int t = 0;
+      auto mma4 = [&](uint32_t d_tmem, uint32_t first_acc) {
+#pragma unroll
+        for (int k4 = 0; k4 < kStageKBytes / kUmmaKBytes; ++k4) {
+          // advancing the start address by 32 bytes (2 units) steps along K inside the swizzle atom
+          const uint64_t da = ((uint64_t)kDescHi << 32) | (uint64_t)(lo + 2u * k4);
+          const uint64_t db = ((uint64_t)kDescHi << 32) | (uint64_t)(lo + kBOff + 2u * k4);
+          const uint32_t acc = k4 == 0 ? first_acc : 1u;
+          if (PAIR) tc_mma_pair<BF16>(d_tmem, da, db, p.idesc, acc);
+          else tc_mma<BF16>(d_tmem, da, db, p.idesc, acc);
+        }
+      };
       for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
         const int a = t & 1;
         if (!mbar_wait(tempty0 + 8 * a, ((t >> 1) & 1) ^ 1, abort_flag, p.err)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)a * kAccCols;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.err)) { ok = false; break; }
+          if (!mbar_wait(fb, ph, abort_flag, p.err)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(stage_base + (size_t)s * stage_bytes);
-          const uint64_t da = smem_desc(a_addr), db = smem_desc(a_addr + BM * kStageKBytes);
-#pragma unroll
-          for (int k4 = 0; k4 < kStageKBytes / kUmmaKBytes; ++k4) {
-            // advancing the start address by 32 bytes (2 units) steps along K inside the swizzle atom
-            if (PAIR) tc_mma_pair<BF16>(d_tmem, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), p.idesc, (kb | k4) != 0);
-            else tc_mma<BF16>(d_tmem, da + (uint64_t)(2 * k4), db + (uint64_t)(2 * k4), p.idesc, (kb | k4) != 0);
-          }
-          if (PAIR) tc_commit_pair(empty0 + 8 * s); else tc_commit(empty0 + 8 * s);   // stage reusable once these MMAs have read it
-          if (++s == p.stages) { s = 0; ph ^= 1; }
+          mma4(d_tmem, kb != 0);
+          // stage reusable once these MMAs have read it
+          if (PAIR) tc_commit_pair(fb + 8 * kMaxStages); else tc_commit(fb + 8 * kMaxStages);
+          lo += lo_step; fb += 8;
+          if (++s == p.stages) { s = 0; ph ^= 1; lo = lo0; fb = full0; }
         }
         if (ok) { if (PAIR) tc_commit_pair(tfull0 + 8 * a); else tc_commit(tfull0 + 8 * a); }   // accumulator complete
       }
