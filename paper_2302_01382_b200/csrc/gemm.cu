@@ -106,6 +106,37 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// The same wait for a whole converged warp, written so that the compiler sees warp-uniform control
+// flow (the spin is inside one asm statement, the outcome is a vote): the producer and the MMA
+// issuer run their loops on all 32 lanes, which keeps their address and descriptor arithmetic on
+// the uniform datapath, and elect one lane only for the TMA / MMA instructions themselves.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* err) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 64;\n\t"
+      "SPIN:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra DONE;\n\t"
+      "sub.u32 n, n, 1;\n\t"
+      "setp.ne.u32 p, n, 0;\n\t"
+      "@p bra SPIN;\n\t"
+      "mov.u32 %0, 0;\n\t"
+      "bra OUT;\n\t"
+      "DONE:\n\t"
+      "mov.u32 %0, 1;\n\t"
+      "OUT:\n\t}"
+      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+  if (__all_sync(0xffffffffu, done != 0)) return true;
+  const bool ok = mbar_wait(bar, parity, abort_flag, err);
+  return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ bool elect_one() {
+  uint32_t e;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(e));
+  return e != 0;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t x, int32_t y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -412,7 +443,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     ld_yb = tn * p.bn + rank * b_rows;
   };
   set_tile_coords();
-  auto issue_load = [&]() {   // the stage's empty barrier must already have been passed
+  const bool elected = elect_one();    // the lane of a converged warp that issues TMA / MMA instructions
+  auto issue_load = [&]() {   // whole warp 0; the stage's empty barrier must already have been passed
+    if (elected) {
     if (PAIR) {
       // the first CTA's barrier collects the bytes of both CTAs' loads
       if (rank == 0) mbar_expect_tx(ld_bar, 2 * stage_bytes);
@@ -422,6 +455,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       mbar_expect_tx(ld_bar, stage_bytes);
       tma_load_2d(ld_dst, &map_a, ld_bar, ld_x, ld_ya);
       tma_load_2d(ld_dst + BM * kStageKBytes, &map_b, ld_bar, ld_x, ld_yb);
+    }
     }
     ld_dst += stage_bytes; ld_bar += 8; ld_x += k_elems;
     if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; ld_dst = stage0; ld_bar = full0; }
@@ -452,7 +486,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   // Everything above touches no global memory, so under programmatic dependent launch it
   // overlaps the tail of the previous kernel in the stream; from here on its results are needed.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (threadIdx.x == 0) {
+  if (warp == 0) {
     // the ring is empty: fill it before the block-wide barrier so the first tiles are in flight
     for (int i = 0; i < p.stages && ld_tile < num_tiles; ++i) issue_load();
   }
@@ -464,29 +498,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      bool ok = true;
-      while (ld_tile < num_tiles) {
-        if (!mbar_wait(ld_bar + 8 * kMaxStages, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
-        issue_load();
+    bool ok = true;
+    while (ld_tile < num_tiles) {
+      if (!mbar_wait_warp(ld_bar + 8 * kMaxStages, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
+      issue_load();
+    }
+    if (PAIR && ok) {
+      // the peer's MMA completions still arrive on this CTA's stage barriers: drain them all
+      // before this CTA may exit (a stage never filled passes at once)
+      for (int i = 0; i < p.stages && ok; ++i) {
+        if (!mbar_wait_warp(empty0 + 8 * ld_s, ld_ph ^ 1, abort_flag, p.err)) ok = false;
+        if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; }
       }
-      if (PAIR && ok) {
-        // the peer's MMA completions still arrive on this CTA's stage barriers: drain them all
-        // before this CTA may exit (a stage never filled passes at once)
-        for (int i = 0; i < p.stages && ok; ++i) {
-          if (!mbar_wait(empty0 + 8 * ld_s, ld_ph ^ 1, abort_flag, p.err)) ok = false;
-          if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; }
-        }
-      }
-      if (!ok) {
-        // give copies already in flight a bounded time to land before the CTA exits
-        const uint64_t t0 = global_timer();
-        while (global_timer() - t0 < 200000ull) {}
-      }
+    }
+    if (!ok) {
+      // give copies already in flight a bounded time to land before the CTA exits
+      const uint64_t t0 = global_timer();
+      while (global_timer() - t0 < 200000ull) {}
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
       // Descriptor low words (start address field, 16-byte units) of the four K steps of the
       // current stage's A and B tiles; the high word is the same for all.
       constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
@@ -498,6 +530,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       bool ok = true;
       int t = 0;
       auto mma4 = [&](uint32_t d_tmem, uint32_t first_acc) {
+        if (!elected) return;
 #pragma unroll
         for (int k4 = 0; k4 < kStageKBytes / kUmmaKBytes; ++k4) {
           // advancing the start address by 32 bytes (2 units) steps along K inside the swizzle atom
@@ -510,19 +543,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       };
       for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
         const int a = t & 1;
-        if (!mbar_wait(tempty0 + 8 * a, ((t >> 1) & 1) ^ 1, abort_flag, p.err)) { ok = false; break; }
+        if (!mbar_wait_warp(tempty0 + 8 * a, ((t >> 1) & 1) ^ 1, abort_flag, p.err)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)a * kAccCols;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait(fb, ph, abort_flag, p.err)) { ok = false; break; }
+          if (!mbar_wait_warp(fb, ph, abort_flag, p.err)) { ok = false; break; }
           tc_fence_after();
           mma4(d_tmem, kb != 0);
           // stage reusable once these MMAs have read it
-          if (PAIR) tc_commit_pair(fb + 8 * kMaxStages); else tc_commit(fb + 8 * kMaxStages);
+          if (elected) { if (PAIR) tc_commit_pair(fb + 8 * kMaxStages); else tc_commit(fb + 8 * kMaxStages); }
           lo += lo_step; fb += 8;
           if (++s == p.stages) { s = 0; ph ^= 1; lo = lo0; fb = full0; }
         }
-        if (ok) { if (PAIR) tc_commit_pair(tfull0 + 8 * a); else tc_commit(tfull0 + 8 * a); }   // accumulator complete
+        if (ok && elected) { if (PAIR) tc_commit_pair(tfull0 + 8 * a); else tc_commit(tfull0 + 8 * a); }   // accumulator complete
       }
     }
   } else {
