@@ -425,6 +425,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // first tile of this CTA (pair)
   const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int rows_per_tile = PAIR ? 2 * BM : BM;
+  // Tiles are numbered with the row-tile index fastest.  Each role walks its tiles by adding the
+  // stride split into (row tiles, column tiles) once here: a division per tile would sit on the
+  // epilogue's and the producer's path.
+  const int step_tn = tile_step / p.tiles_m, step_tm = tile_step - step_tn * p.tiles_m;
+  const int tm0 = tile0 % p.tiles_m, tn0 = tile0 / p.tiles_m;
 
   // producer state (thread 0 only): next k-block to load
   // The producer and the MMA issuer share their scheduler with four epilogue warps that almost
@@ -437,10 +442,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const uint32_t stage0 = smem_u32(stage_base);
   uint32_t ld_dst = stage0, ld_bar = full0;      // stage address and its full barrier
   int ld_x = 0, ld_ya = 0, ld_yb = 0;            // TMA coordinates of the next k-block
+  int ld_tm = tm0, ld_tn = tn0;
   auto set_tile_coords = [&]() {
-    const int tm = ld_tile % p.tiles_m, tn = ld_tile / p.tiles_m;
-    ld_ya = tm * rows_per_tile + rank * BM;
-    ld_yb = tn * p.bn + rank * b_rows;
+    ld_ya = ld_tm * rows_per_tile + rank * BM;
+    ld_yb = ld_tn * p.bn + rank * b_rows;
   };
   set_tile_coords();
   const bool elected = elect_one();    // the lane of a converged warp that issues TMA / MMA instructions
@@ -459,7 +464,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
     ld_dst += stage_bytes; ld_bar += 8; ld_x += k_elems;
     if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; ld_dst = stage0; ld_bar = full0; }
-    if (++ld_kb == p.k_blocks) { ld_kb = 0; ld_x = 0; ld_tile += tile_step; set_tile_coords(); }
+    if (++ld_kb == p.k_blocks) {
+      ld_kb = 0; ld_x = 0; ld_tile += tile_step;
+      ld_tm += step_tm; ld_tn += step_tn;
+      if (ld_tm >= p.tiles_m) { ld_tm -= p.tiles_m; ++ld_tn; }
+      set_tile_coords();
+    }
   };
 
   if (threadIdx.x == 0) {
@@ -571,21 +581,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     uint32_t cursor = 0;
     bool ok = true;
     int t = 0;
+    // Weight scales of this warp's chunks, one column per lane and chunk.  They are fetched one
+    // tile ahead: when the epilogue is the longer phase the accumulator is already waiting at
+    // the top of the loop, and a load issued there would put its whole latency on the tile.
+    auto load_scales = [&](int tile, int tile_tn, float (&w)[2]) {
+      w[0] = 0.f; w[1] = 0.f;
+      if (BF16 || !p.need_y || tile >= num_tiles) return;
+      const int cb = tile_tn * p.bn + c_begin * 32;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int col = cb + j * 32 + lane;
+        if (c_begin + j < c_end && col < p.n) w[j] = __ldg(p.scale_w + col);
+      }
+    };
+    float sw_next[2];
+    load_scales(tile0, tn0, sw_next);
+    int tm = tm0, tn = tn0;
     for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
       const int a = t & 1;
-      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
       const int row0 = tm * rows_per_tile + rank * BM + quad * 32;
       const int col_base = tn * p.bn + c_begin * 32;
-      // column scales of this warp's chunks, one column per lane and chunk, fetched while the
-      // tensor cores are still working on the tile
-      float cs[2] = {0.f, 0.f};
-      if (!BF16 && p.need_y) {
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const int col = col_base + j * 32 + lane;
-          if (c_begin + j < c_end && col < p.n) cs[j] = __fmul_rn(p.scale_x, __ldg(p.scale_w + col));
-        }
-      }
+      const float cs[2] = {__fmul_rn(p.scale_x, sw_next[0]), __fmul_rn(p.scale_x, sw_next[1])};
+      int tm_next = tm + step_tm, tn_next = tn + step_tn;
+      if (tm_next >= p.tiles_m) { tm_next -= p.tiles_m; ++tn_next; }
+      load_scales(tile + tile_step, tn_next, sw_next);
       if (!mbar_wait(tfull0 + 8 * a, (t >> 1) & 1, abort_flag, p.err)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * kAccCols + c_begin * 32);
@@ -608,6 +627,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         __syncwarp();
         if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
       }
+      tm = tm_next; tn = tn_next;
     }
     // all TMA stores of this warp must have completed before the CTA's shared memory goes away
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
