@@ -225,6 +225,24 @@ int qcfg_model_weight_absmax(qcfg_model* model, int32_t layer, float* absmax_hos
 int qcfg_eval_config(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits,
                      const float* x_dev, int64_t m, float* const* y_dev, void* stream);
 
+/* Latency table of Section 4, "Compute Latency Estimates": the paper prices a configuration by
+ * benchmarking every layer's kernel at every available precision and adding up the entries the
+ * configuration selects.  For each bs[i] (values in {2..8, 16}) the model is run with every
+ * layer at that width, `reps` times after one untimed pass, with a CUDA event pair around all
+ * the kernels each layer launches (operand preparation and GEMM with its fused epilogue; codes
+ * a producer writes for its consumer count towards the producer).  ms_host is a HOST array
+ * [n_layers][n_bs] of mean milliseconds.  Synchronises the stream after every pass; event
+ * pairs serialise the launches, so a column's sum exceeds the time of one untimed evaluation.
+ * On this hardware every integer width 2..8 runs on the same int8 tensor path.               */
+int qcfg_latency_table(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int64_t m,
+                       const uint8_t* bs, int32_t n_bs, int32_t reps, float* ms_host, void* stream);
+/* The two deployment costs the searches minimise (Table 1 rows "Size" and "Latency"): size =
+ * sum over layers of n_out * k_in * bits[l] / 8 bytes (weights only); latency = sum over layers of
+ * the table entry of (l, bits[l]).  Host only.  latency_ms or size_bytes may be NULL; without
+ * latency_ms the table arguments are ignored.  A bit width absent from bs gives QCFG_EBITS.  */
+int qcfg_config_cost(qcfg_model* model, const uint8_t* bits, const uint8_t* bs, int32_t n_bs,
+                     const float* ms_host, double* latency_ms, double* size_bytes);
+
 /* The paper's two configuration searches as host drivers over qcfg_eval_config.
  * QCFG_SEARCH_BISECTION is Algorithm 1, QCFG_SEARCH_GREEDY Algorithm 2.  order[n_layers] lists
  * the layers by ascending sensitivity (e.g. the E_QE ranking from qcfg_quant_error_sweep);

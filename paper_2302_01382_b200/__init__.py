@@ -26,7 +26,7 @@ EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error",
            "qcfg_set_fusion", "qcfg_set_pair_tiles", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
-           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_search", "qcfg_debug_dump"]
+           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_latency_table", "qcfg_config_cost", "qcfg_search", "qcfg_debug_dump"]
 
 
 class QcfgError(RuntimeError):
@@ -81,6 +81,9 @@ def load_library() -> C.CDLL:
         "qcfg_debug_dump": [vp, vp, i32, vp, vp, vp, vp],
         "qcfg_search": [vp, vp, ci, C.POINTER(i32), C.POINTER(C.c_uint8), i32, C.c_double, vp, i64, C.POINTER(C.c_uint8),
                         C.POINTER(C.c_uint8), C.POINTER(C.c_double), i32, C.POINTER(i32), vp],
+        "qcfg_latency_table": [vp, vp, vp, i64, C.POINTER(C.c_uint8), i32, i32, C.POINTER(C.c_float), vp],
+        "qcfg_config_cost": [vp, C.POINTER(C.c_uint8), C.POINTER(C.c_uint8), i32, C.POINTER(C.c_float), C.POINTER(C.c_double),
+                             C.POINTER(C.c_double)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -307,6 +310,28 @@ class Model:
         k = min(n_evals.value, capacity)
         vis = [list(visited[i * n:(i + 1) * n]) for i in range(k)]
         return list(bits), vis, list(acc[:k]), n_evals.value
+
+    def latency_table(self, x: torch.Tensor, m: int, bs, reps: int = 5, stream=None):
+        """Mean milliseconds of every layer at every width of bs: list of n_layers rows of len(bs) floats."""
+        n = len(self.layers)
+        bs_a = (C.c_uint8 * len(bs))(*[int(v) for v in bs])
+        out = (C.c_float * (n * len(bs)))()
+        self.ctx._check(self.ctx.lib.qcfg_latency_table(self.ctx.h, self.h, _ptr(x), m, bs_a, len(bs), reps, out, _stream(stream)))
+        return [list(out[l * len(bs):(l + 1) * len(bs)]) for l in range(n)]
+
+    def config_cost(self, bits, bs=None, table=None):
+        """(latency in ms or None, size in bytes) of a configuration; latency needs bs and the table."""
+        n = len(self.layers)
+        b = (C.c_uint8 * n)(*[int(v) for v in bits])
+        size = C.c_double()
+        if table is None:
+            self.ctx._check(self.ctx.lib.qcfg_config_cost(self.h, b, None, 0, None, None, C.byref(size)))
+            return None, size.value
+        bs_a = (C.c_uint8 * len(bs))(*[int(v) for v in bs])
+        flat = (C.c_float * (n * len(bs)))(*[float(v) for row in table for v in row])
+        lat = C.c_double()
+        self.ctx._check(self.ctx.lib.qcfg_config_cost(self.h, b, bs_a, len(bs), flat, C.byref(lat), C.byref(size)))
+        return lat.value, size.value
 
     def debug_dump(self, layer: int, qx: Optional[torch.Tensor], qw: Optional[torch.Tensor], acc: Optional[torch.Tensor], stream=None):
         self.ctx._check(self.ctx.lib.qcfg_debug_dump(self.ctx.h, self.h, layer, _ptr(qx), _ptr(qw), _ptr(acc), _stream(stream)))

@@ -233,7 +233,7 @@ int64_t ext_ld_of(const Model* M) {
 
 // One forward pass.  calibrate = true: every layer at 16 bit, record max|input| per layer.
 int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t x_ld, int64_t m,
-            float* const* y_dev, bool calibrate, cudaStream_t st) {
+            float* const* y_dev, bool calibrate, cudaStream_t st, cudaEvent_t* layer_ev = nullptr) {
   const int n = (int)M->L.size();
   for (int l = 0; l < n; ++l) {
     LayerState& S = M->L[l];
@@ -247,6 +247,8 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     const int b = S.bits;
     int rc = ensure_weight_codes(ctx, S, b, st);
     if (rc) return rc;
+    // optional per-layer timing: everything this layer launches (operand preparation and GEMM)
+    if (layer_ev && cudaEventRecord(layer_ev[2 * l], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
 
     // ---- GEMM input codes
     if (!S.a_ready) {
@@ -379,6 +381,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     }
     rc = launch_gemm(ctx, g, st);
     if (rc) return rc;
+    if (layer_ev && cudaEventRecord(layer_ev[2 * l + 1], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
   }
   return QCFG_OK;
 }
@@ -707,6 +710,71 @@ int qcfg_eval_config(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, cons
   if (rc) return rc;
   M->evaluated = true;
   M->last_m = m;
+  return QCFG_OK;
+}
+
+// ---- latency table and configuration cost (Section 4, "Compute Latency Estimates"; Table 1) ----
+
+int qcfg_latency_table(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int64_t m, const uint8_t* bs, int32_t n_bs,
+                       int32_t reps, float* ms_host, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  if (!x_dev || !bs || !ms_host || m <= 0 || n_bs <= 0 || reps <= 0) return set_error(c, QCFG_EINVAL, "latency_table: null pointer or non-positive count");
+  if (!M->calibrated) return set_error(c, QCFG_ESTATE, "latency_table: model is not calibrated");
+  if ((uintptr_t)x_dev % 4) return set_error(c, QCFG_EALIGN, "latency_table: x_dev not 4-byte aligned");
+  for (int i = 0; i < n_bs; ++i)
+    if (!bits_ok(bs[i])) return set_error(c, QCFG_EBITS, "latency_table: bs[%d] = %d", i, (int)bs[i]);
+  const int n = (int)M->L.size();
+  cudaStream_t st = (cudaStream_t)stream;
+  std::vector<cudaEvent_t> ev((size_t)2 * n, nullptr);
+  int rc = QCFG_OK;
+  for (auto& e : ev)
+    if (rc == QCFG_OK && cudaEventCreate(&e) != cudaSuccess) rc = set_error(c, QCFG_ECUDA, "latency_table: cudaEventCreate failed");
+  std::vector<uint8_t> bits((size_t)n);
+  std::vector<double> sum((size_t)n);
+  const int64_t ext_ld = ext_ld_of(M);
+  for (int i = 0; i < n_bs && rc == QCFG_OK; ++i) {
+    std::fill(bits.begin(), bits.end(), bs[i]);
+    std::fill(sum.begin(), sum.end(), 0.0);
+    rc = forward(c, M, bits.data(), x_dev, ext_ld, m, nullptr, false, st);        // fills the weight-code cache
+    for (int r = 0; r < reps && rc == QCFG_OK; ++r) {
+      rc = forward(c, M, bits.data(), x_dev, ext_ld, m, nullptr, false, st, ev.data());
+      if (rc == QCFG_OK) rc = check_cuda(c, cudaEventSynchronize(ev[(size_t)2 * n - 1]), "latency_table: event synchronize");
+      for (int l = 0; l < n && rc == QCFG_OK; ++l) {
+        float ms = 0.f;
+        rc = check_cuda(c, cudaEventElapsedTime(&ms, ev[2 * l], ev[2 * l + 1]), "latency_table: elapsed time");
+        sum[l] += ms;
+      }
+    }
+    if (rc == QCFG_OK)
+      for (int l = 0; l < n; ++l) ms_host[(size_t)l * n_bs + i] = (float)(sum[l] / reps);
+  }
+  for (auto& e : ev) if (e) cudaEventDestroy(e);
+  if (rc == QCFG_OK) { M->evaluated = true; M->last_m = m; }
+  return rc;
+}
+
+int qcfg_config_cost(qcfg_model* model, const uint8_t* bits, const uint8_t* bs, int32_t n_bs, const float* ms_host,
+                     double* latency_ms, double* size_bytes) {
+  if (!model || !bits) return QCFG_EINVAL;
+  Model* M = &model->m;
+  Ctx* c = M->ctx;
+  if (latency_ms && (!bs || !ms_host || n_bs <= 0)) return set_error(c, QCFG_EINVAL, "config_cost: latency wanted without a table");
+  const int n = (int)M->L.size();
+  double lat = 0.0, size = 0.0;
+  for (int l = 0; l < n; ++l) {
+    if (!bits_ok(bits[l])) return set_error(c, QCFG_EBITS, "config_cost: layer %d has bit width %d", l, (int)bits[l]);
+    size += (double)M->L[l].d.n_out * (double)M->L[l].d.k_in * (double)bits[l] / 8.0;
+    if (latency_ms) {
+      int col = -1;
+      for (int i = 0; i < n_bs; ++i) if (bs[i] == bits[l]) col = i;
+      if (col < 0) return set_error(c, QCFG_EBITS, "config_cost: layer %d uses %d bit, which the table does not cover", l, (int)bits[l]);
+      lat += (double)ms_host[(size_t)l * n_bs + col];
+    }
+  }
+  if (latency_ms) *latency_ms = lat;
+  if (size_bytes) *size_bytes = size;
   return QCFG_OK;
 }
 

@@ -30,6 +30,7 @@ def main():
     ap.add_argument("--seed", type=int, default=2)
     ap.add_argument("--resnet", type=int, default=0, help="batch size: run the ResNet-50 table instead of a BERT stack")
     ap.add_argument("--mixed", action="store_true", help="use the workload's drawn bit configuration instead of --bits")
+    ap.add_argument("--latency", type=int, default=0, help="repetitions: print the per-width latency table sums and model sizes")
     ap.add_argument("--single-cta", action="store_true", help="128-row GEMM tiles on one CTA each instead of CTA pairs")
     args = ap.parse_args()
 
@@ -59,6 +60,13 @@ def main():
     ctx.check_sync()
     print(f"evaluations: host enqueue {1e3 * t_host / args.evals:.3f} ms, device {e0.elapsed_time(e1) / args.evals:.3f} ms each "
           f"({len(w.layers)} layers, m = {w.m}, bits {sorted(set(int(b) for b in bits))})")
+    if args.latency:
+        bs = [16, 8, 4]
+        table = model.latency_table(x, w.m, bs, reps=args.latency)
+        ctx.check_sync()
+        for i, b in enumerate(bs):
+            lat, size = model.config_cost([b] * len(w.layers), bs, table)
+            print(f"all layers at {b:2d} bit: summed layer latency {lat:.3f} ms, weights {size / 1e6:.2f} MB")
     if args.sweep:
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         sse, amax = ctx.quant_error_sweep(weights, PER_ROW)

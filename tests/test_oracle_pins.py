@@ -13,6 +13,7 @@ import torch
 
 import qcfg_workloads as wl
 from oracle import qcfg_oracle as orc
+from oracle import cost_oracle as cost
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 BITS = list(range(2, 9))
@@ -339,6 +340,21 @@ def test_layer_tables_match_table1_sizes():
     for model, b, mb in _golden("table1_sizes.txt"):
         L = tables[model]
         assert wl.size_mb(L, [int(b)] * len(L)) == pytest.approx(float(mb), abs=0.0075)
+        assert cost.size_bytes(L, [int(b)] * len(L)) / 1e6 == pytest.approx(float(mb), abs=0.0075)
+
+
+def test_cost_oracle_latency_is_the_selected_entries_sum_and_size_is_linear_in_bits():
+    L = wl.mlp_layers([256, 256, 256, 10])
+    table = [[1.0, 2.0, 4.0], [8.0, 16.0, 32.0], [64.0, 128.0, 256.0]]      # distinct powers of two: the sum names its terms
+    assert cost.latency_ms(table, [4, 8, 16], [4, 8, 16]) == 1.0 + 16.0 + 256.0
+    assert cost.latency_ms(table, [4, 8, 16], [16, 4, 8]) == 4.0 + 8.0 + 128.0
+    assert cost.latency_ms(table, [16, 8, 4], [4, 4, 4]) == 4.0 + 32.0 + 256.0    # columns follow bs, not the width
+    with pytest.raises(KeyError):
+        cost.latency_ms(table, [4, 8, 16], [4, 2, 16])
+    # hand count: 256*256 + 256*256 + 10*256 parameters
+    assert cost.size_bytes(L, [8, 8, 8]) == 256 * 256 * 2 + 2560
+    assert cost.size_bytes(L, [4, 8, 16]) == 256 * 256 * 0.5 + 256 * 256 + 2560 * 2
+    assert cost.size_bytes(L, [2, 2, 2]) * 8 == cost.size_bytes(L, [16, 16, 16])
 
 
 def test_search_sequences_follow_the_algorithms():
