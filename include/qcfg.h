@@ -243,6 +243,20 @@ int qcfg_latency_table(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int
 int qcfg_config_cost(qcfg_model* model, const uint8_t* bits, const uint8_t* bs, int32_t n_bs,
                      const float* ms_host, double* latency_ms, double* size_bytes);
 
+/* Noise-injection sensitivity E_N (Section 3.1, Eqs. 3-5): for each layer i in turn, Gaussian
+ * noise nu = sigma_i * noise_dev[i], sigma_i = lambda * max|w_i| (whole tensor), is added to that
+ * layer's weights only, the model is run on x_dev and E_N(i) = L(x, W*) - L(x, W).  The loss needs
+ * labels the library does not have: L is the relative distance ||y - y_0||_2 / ||y_0||_2 of the last
+ * layer's fp32 output from the noise-free output y_0, so L(x, W) = 0.  The model runs with every
+ * layer at 16 bit (the paper's floating-point baseline; the perturbed weights are rounded to bf16
+ * like the clean ones).  The second argument of N(0, .) is read as the standard deviation.
+ * noise_dev is a HOST array of n_layers DEVICE pointers to the caller's standard-normal draws,
+ * [n_out x k_in] row-major like the weights (the generator is the caller's); a NULL entry skips
+ * the layer (E_N = 0).  e_n_host receives n_layers doubles.  Costs one forward per perturbed layer
+ * plus one; synchronises the stream after each.  No calibration needed.                        */
+int qcfg_noise_sensitivity(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int64_t m,
+                           const float* const* noise_dev, float lambda, double* e_n_host, void* stream);
+
 /* The paper's two configuration searches as host drivers over qcfg_eval_config.
  * QCFG_SEARCH_BISECTION is Algorithm 1, QCFG_SEARCH_GREEDY Algorithm 2.  order[n_layers] lists
  * the layers by ascending sensitivity (e.g. the E_QE ranking from qcfg_quant_error_sweep);

@@ -26,7 +26,7 @@ EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error",
            "qcfg_set_fusion", "qcfg_set_pair_tiles", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
-           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_latency_table", "qcfg_config_cost", "qcfg_search", "qcfg_debug_dump"]
+           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_latency_table", "qcfg_config_cost", "qcfg_noise_sensitivity", "qcfg_search", "qcfg_debug_dump"]
 
 
 class QcfgError(RuntimeError):
@@ -81,6 +81,7 @@ def load_library() -> C.CDLL:
         "qcfg_debug_dump": [vp, vp, i32, vp, vp, vp, vp],
         "qcfg_search": [vp, vp, ci, C.POINTER(i32), C.POINTER(C.c_uint8), i32, C.c_double, vp, i64, C.POINTER(C.c_uint8),
                         C.POINTER(C.c_uint8), C.POINTER(C.c_double), i32, C.POINTER(i32), vp],
+        "qcfg_noise_sensitivity": [vp, vp, vp, i64, C.POINTER(C.c_void_p), C.c_float, C.POINTER(C.c_double), vp],
         "qcfg_latency_table": [vp, vp, vp, i64, C.POINTER(C.c_uint8), i32, i32, C.POINTER(C.c_float), vp],
         "qcfg_config_cost": [vp, C.POINTER(C.c_uint8), C.POINTER(C.c_uint8), i32, C.POINTER(C.c_float), C.POINTER(C.c_double),
                              C.POINTER(C.c_double)],
@@ -310,6 +311,14 @@ class Model:
         k = min(n_evals.value, capacity)
         vis = [list(visited[i * n:(i + 1) * n]) for i in range(k)]
         return list(bits), vis, list(acc[:k]), n_evals.value
+
+    def noise_sensitivity(self, x: torch.Tensor, m: int, noises, lam: float, stream=None):
+        """E_N per layer (Eqs. 3-5); noises[l] is a standard-normal tensor shaped like layer l's weight, or None."""
+        n = len(self.layers)
+        ptrs = (C.c_void_p * n)(*[None if t is None else t.data_ptr() for t in noises])
+        out = (C.c_double * n)()
+        self.ctx._check(self.ctx.lib.qcfg_noise_sensitivity(self.ctx.h, self.h, _ptr(x), m, ptrs, float(lam), out, _stream(stream)))
+        return list(out)
 
     def latency_table(self, x: torch.Tensor, m: int, bs, reps: int = 5, stream=None):
         """Mean milliseconds of every layer at every width of bs: list of n_layers rows of len(bs) floats."""

@@ -163,6 +163,7 @@ struct Model {
   bool evaluated = false;
   DevBuf act_absmax_dev;           // fp32 [n_layers], filled by calibration
   DevBuf search_ref, search_out, search_partial;   // buffers of the search drivers
+  DevBuf noise_codes, noise_amax;                  // perturbed bf16 weights of one layer and its max|w|
   int64_t last_m = 0;
 };
 
@@ -891,6 +892,66 @@ int qcfg_search(qcfg_ctx* ctx, qcfg_model* model, int algorithm, const int32_t* 
   }
   memcpy(bits_out, w.data(), n);
   if (n_evals) *n_evals = S.evals;
+  return QCFG_OK;
+}
+
+// ---- noise-injection sensitivity E_N (Section 3.1, Eqs. 3-5) ----------------------------------
+
+int qcfg_noise_sensitivity(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, int64_t m, const float* const* noise_dev,
+                           float lambda, double* e_n_host, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  const int n = (int)M->L.size();
+  if (!x_dev || !noise_dev || !e_n_host || m <= 0) return set_error(c, QCFG_EINVAL, "noise_sensitivity: null pointer or m <= 0");
+  if (!(lambda >= 0.0f) || !std::isfinite(lambda)) return set_error(c, QCFG_EINVAL, "noise_sensitivity: lambda must be finite and >= 0");
+  if ((uintptr_t)x_dev % 4) return set_error(c, QCFG_EALIGN, "noise_sensitivity: x_dev not 4-byte aligned");
+  for (int l = 0; l < n; ++l)
+    if (noise_dev[l] && (uintptr_t)noise_dev[l] % 4) return set_error(c, QCFG_EALIGN, "noise_sensitivity: noise_dev[%d] not 4-byte aligned", l);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t out_elems = layer_rows(M, n - 1, m) * M->L[n - 1].d.n_out;
+  const int blocks = c->sms * 4;
+  size_t code_bytes = 0;
+  for (auto& S : M->L) code_bytes = std::max(code_bytes, (size_t)(S.d.n_out * S.ldk) * 2);
+  int rc = M->search_ref.ensure(c, (size_t)out_elems * 4);
+  if (!rc) rc = M->search_out.ensure(c, (size_t)out_elems * 4);
+  if (!rc) rc = M->search_partial.ensure(c, (size_t)blocks * 16);
+  if (!rc) rc = M->noise_codes.ensure(c, code_bytes);
+  if (!rc) rc = M->noise_amax.ensure(c, 4);
+  if (rc) return rc;
+  std::vector<double> partial((size_t)blocks * 2);
+  std::vector<uint8_t> bits((size_t)n, 16);
+  std::vector<float*> ys((size_t)n, nullptr);
+  const int64_t ext_ld = ext_ld_of(M);
+  // the noise-free model: every layer at 16 bit
+  ys[n - 1] = (float*)M->search_ref.p;
+  rc = forward(c, M, bits.data(), x_dev, ext_ld, m, ys.data(), false, st);
+  if (rc) return rc;
+  ys[n - 1] = (float*)M->search_out.p;
+  for (int i = 0; i < n; ++i) {
+    e_n_host[i] = 0.0;
+    if (!noise_dev[i]) continue;
+    LayerState& S = M->L[i];
+    rc = launch_absmax(c, S.d.w_dev, S.d.n_out, S.d.k_in, S.d.k_in, QCFG_PER_TENSOR, (float*)M->noise_amax.p, st);
+    if (!rc) rc = launch_perturb_bf16(c, S.d.w_dev, noise_dev[i], (const float*)M->noise_amax.p, lambda, S.d.n_out, S.d.k_in,
+                                      M->noise_codes.p, S.ldk, st);
+    if (rc) return rc;
+    void* clean = S.wc[16].codes.p;               // W* = W without w_i, plus w_i + nu
+    S.wc[16].codes.p = M->noise_codes.p;
+    rc = forward(c, M, bits.data(), x_dev, ext_ld, m, ys.data(), false, st);
+    S.wc[16].codes.p = clean;
+    if (!rc) rc = launch_sqdiff(c, (const float*)M->search_out.p, (const float*)M->search_ref.p, out_elems,
+                                (double*)M->search_partial.p, blocks, st);
+    if (!rc) rc = check_cuda(c, cudaMemcpyAsync(partial.data(), M->search_partial.p, (size_t)blocks * 16, cudaMemcpyDeviceToHost, st),
+                             "noise_sensitivity: copy");
+    if (!rc) rc = qcfg_sync_status(ctx, st);
+    if (rc) return rc;
+    double d2 = 0.0, r2 = 0.0;
+    for (int b = 0; b < blocks; ++b) { d2 += partial[2 * b]; r2 += partial[2 * b + 1]; }
+    e_n_host[i] = r2 > 0.0 ? std::sqrt(d2 / r2) : (d2 == 0.0 ? 0.0 : INFINITY);
+  }
+  M->evaluated = true;
+  M->last_m = m;
   return QCFG_OK;
 }
 

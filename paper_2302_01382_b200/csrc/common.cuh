@@ -42,6 +42,8 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
                     const float* inv_scale_ptr, float inv_scale_val, int granularity, int bits,
                     void* q, int64_t ldq, cudaStream_t st);
 
+int launch_perturb_bf16(Ctx* ctx, const float* w, const float* nu, const float* amax_dev, float lambda, int64_t rows,
+                        int64_t cols, void* q, int64_t ldq, cudaStream_t st);
 int launch_sqdiff(Ctx* ctx, const float* y, const float* ref, int64_t n, double* partial, int blocks, cudaStream_t st);
 
 // ----- conv.cu ------------------------------------------------------------------------

@@ -213,6 +213,37 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
 }
 
 
+// ------------------------------------------------------------------------------- noise injection (Eqs. 3-5)
+
+// bf16 operand of a weight tensor with Gaussian noise added: w + (lambda * max|w|) * nu, nu being
+// the caller's standard-normal draws; one fp32 multiply for the deviation, one for the scaled
+// draw, one add (no FMA), then round-to-nearest-even to bf16.  Columns cols..ldq-1 are zero.
+__global__ void __launch_bounds__(256) perturb_bf16_kernel(const float* __restrict__ w, const float* __restrict__ nu,
+                                                           const float* __restrict__ amax, float lambda, int64_t rows,
+                                                           int64_t cols, __nv_bfloat16* __restrict__ q, int64_t ldq) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * ldq) return;
+  const int64_t r = idx / ldq, c = idx - r * ldq;
+  float v = 0.0f;
+  if (c < cols) {
+    const float sigma = __fmul_rn(lambda, __ldg(amax));
+    v = __fadd_rn(__ldg(w + r * cols + c), __fmul_rn(sigma, __ldg(nu + r * cols + c)));
+  }
+  q[idx] = __float2bfloat16_rn(v);
+}
+
+int launch_perturb_bf16(Ctx* ctx, const float* w, const float* nu, const float* amax_dev, float lambda, int64_t rows,
+                        int64_t cols, void* q, int64_t ldq, cudaStream_t st) {
+  const int64_t total = rows * ldq;
+  if (total == 0) return QCFG_OK;
+  prof_begin(ctx, 2, st);
+  perturb_bf16_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(w, nu, amax_dev, lambda, rows, cols,
+                                                                      reinterpret_cast<__nv_bfloat16*>(q), ldq);
+  prof_end(ctx, 2, 0.0, st);
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "perturb launch");
+}
+
 // ------------------------------------------------------------------------------- output fidelity
 
 // Per-block partial sums of (y - ref)^2 and ref^2 in fp64 (fixed grid, fixed order: deterministic).

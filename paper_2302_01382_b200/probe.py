@@ -31,6 +31,7 @@ def main():
     ap.add_argument("--resnet", type=int, default=0, help="batch size: run the ResNet-50 table instead of a BERT stack")
     ap.add_argument("--mixed", action="store_true", help="use the workload's drawn bit configuration instead of --bits")
     ap.add_argument("--latency", type=int, default=0, help="repetitions: print the per-width latency table sums and model sizes")
+    ap.add_argument("--noise", type=float, default=0.0, help="lambda: run the noise-injection sensitivity E_N over all layers")
     ap.add_argument("--single-cta", action="store_true", help="128-row GEMM tiles on one CTA each instead of CTA pairs")
     args = ap.parse_args()
 
@@ -67,6 +68,15 @@ def main():
         for i, b in enumerate(bs):
             lat, size = model.config_cost([b] * len(w.layers), bs, table)
             print(f"all layers at {b:2d} bit: summed layer latency {lat:.3f} ms, weights {size / 1e6:.2f} MB")
+    if args.noise > 0:
+        gen = torch.Generator(device="cuda").manual_seed(args.seed)
+        noises = [torch.randn(t.shape, generator=gen, device="cuda") for t in weights]
+        model.noise_sensitivity(x, w.m, noises, args.noise)           # warm-up (allocations)
+        t0 = time.perf_counter()
+        e_n = model.noise_sensitivity(x, w.m, noises, args.noise)
+        dt = time.perf_counter() - t0
+        print(f"E_N over {len(e_n)} layers at lambda = {args.noise}: {1e3 * dt:.1f} ms ({1e3 * dt / (len(e_n) + 1):.3f} ms per forward), "
+              f"min {min(e_n):.3e} max {max(e_n):.3e}")
     if args.sweep:
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         sse, amax = ctx.quant_error_sweep(weights, PER_ROW)

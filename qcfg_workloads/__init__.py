@@ -259,6 +259,12 @@ def resnet50(seed: int = 3, batch: int = 128, in_hw: int = 224, width: int = 64,
 
 # ------------------------------------------------------------- scripted search sequences
 
+def standard_normal_like(weights, seed: int):
+    """One array of standard-normal draws per weight tensor (the random numbers E_N's noise is built from)."""
+    rng = np.random.default_rng(seed)
+    return [rng.standard_normal(w.shape).astype(np.float32) for w in weights]
+
+
 def greedy_sequence(ranking: Sequence[int], accept: Sequence[bool], start_bits: int = 8,
                     low_bits: int = 4) -> List[np.ndarray]:
     """Configurations visited by one pass of the greedy loop (Algorithm 2, inner loop).
