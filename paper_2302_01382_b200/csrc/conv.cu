@@ -81,7 +81,22 @@ int launch_avgpool(Ctx* ctx, const float* src, int64_t B, int HW, int C, float* 
 
 struct ConvGeom {
   int H, W, C, kh, kw, stride, pad, OH, OW, K;
+  int kwC, WC;                 // elements of one kernel row (kw * C) and of one image row (W * C)
+  uint32_t dm, ds1, ds2;       // division by kwC as multiply-high and shifts
 };
+
+// floor(n / d) for any 32-bit n with the constants of fastdiv_init(d)
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, uint32_t m, uint32_t s1, uint32_t s2) {
+  const uint32_t t = __umulhi(m, n);
+  return (t + ((n - t) >> s1)) >> s2;
+}
+static void fastdiv_init(uint32_t d, uint32_t* m, uint32_t* s1, uint32_t* s2) {
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;                                  // ceil(log2 d)
+  *m = (uint32_t)((((1ull << l) - d) << 32) / d + 1);
+  *s1 = l < 1 ? l : 1;
+  *s2 = l > 0 ? l - 1 : 0;
+}
 
 __device__ __forceinline__ int conv_code(float x, float inv_scale, float qmax) {
   float t = __fmul_rn(x, inv_scale);
@@ -89,63 +104,67 @@ __device__ __forceinline__ int conv_code(float x, float inv_scale, float qmax) {
   return __float2int_rn(t);
 }
 
-// Each thread produces 8 consecutive elements of one row of the [B*OH*OW x ldq] operand.
+// Operand row (b, oh, ow) holds the patch in (kh, kw, cin) order.  For a fixed kernel row dy the kw * C
+// values are contiguous in the NHWC source, so element k = dy * kwC + r comes from offset
+// (ow * stride - pad) * C + r of image row ih = oh * stride - pad + dy, if that offset lies inside the
+// row: one division per group instead of one per index level.  blockIdx.x = b * OH + oh,
+// blockIdx.y and threadIdx.y give ow, threadIdx.x strides over groups of 8 consecutive k.
 template <bool BF16>
-__global__ void __launch_bounds__(256) im2col_quantize_kernel(const float* __restrict__ src, int64_t rows, ConvGeom g,
-                                                              float inv_scale, float qmax, void* __restrict__ q,
-                                                              int64_t ldq, int vec) {
-  const int64_t gpr = ldq >> 3;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * gpr) return;
-  const int64_t row = idx / gpr;
-  const int k0 = (int)((idx - row * gpr) << 3);
-  const int ow = (int)(row % g.OW);
-  const int64_t t = row / g.OW;
-  const int oh = (int)(t % g.OH);
-  const int64_t b = t / g.OH;
-  float v[8];
-  if (vec && k0 + 8 <= g.K) {      // C % 8 == 0: the 8 elements are 8 channels of one tap
-    const int tap = k0 / g.C, c = k0 - tap * g.C;
-    const int dy = tap / g.kw, dx = tap - dy * g.kw;
-    const int ih = oh * g.stride - g.pad + dy, iw = ow * g.stride - g.pad + dx;
-    if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) {
-      const float4* p = reinterpret_cast<const float4*>(src + ((b * g.H + ih) * g.W + iw) * (int64_t)g.C + c);
-      float4 a = __ldg(p), bb = __ldg(p + 1);
-      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = bb.x; v[5] = bb.y; v[6] = bb.z; v[7] = bb.w;
+__global__ void __launch_bounds__(256) im2col_quantize_kernel(const float* __restrict__ src, ConvGeom g, float inv_scale,
+                                                              float qmax, void* __restrict__ q, int64_t ldq, int vec) {
+  const int boh = blockIdx.x;
+  const int b = boh / g.OH, oh = boh - b * g.OH;
+  const int ow = blockIdx.y * blockDim.y + threadIdx.y;
+  if (ow >= g.OW) return;
+  const int64_t row = (int64_t)boh * g.OW + ow;
+  const int off0 = (ow * g.stride - g.pad) * g.C;
+  const int ih0 = oh * g.stride - g.pad;
+  const float* img = src + (int64_t)b * g.H * g.WC;
+  const int gpr = (int)(ldq >> 3);
+  for (int kg = threadIdx.x; kg < gpr; kg += blockDim.x) {
+    const int k0 = kg << 3;
+    float v[8];
+    if (vec) {                       // C % 8 == 0: the 8 elements share dy, dx and validity
+      bool ok = k0 < g.K;
+      const int dy = (int)fastdiv((uint32_t)k0, g.dm, g.ds1, g.ds2);
+      const int off = off0 + (k0 - dy * g.kwC), ih = ih0 + dy;
+      ok = ok && ih >= 0 && ih < g.H && off >= 0 && off < g.WC;
+      if (ok) {
+        const float4* p = reinterpret_cast<const float4*>(img + (int64_t)ih * g.WC + off);
+        const float4 a = __ldg(p), c = __ldg(p + 1);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = 0.0f;
+      }
     } else {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = 0.0f;
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int k = k0 + j;
-      float x = 0.0f;
-      if (k < g.K) {
-        const int tap = k / g.C, c = k - tap * g.C;
-        const int dy = tap / g.kw, dx = tap - dy * g.kw;
-        const int ih = oh * g.stride - g.pad + dy, iw = ow * g.stride - g.pad + dx;
-        if (ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) x = __ldg(src + ((b * g.H + ih) * g.W + iw) * (int64_t)g.C + c);
+      for (int j = 0; j < 8; ++j) {
+        const int k = k0 + j;
+        const int dy = (int)fastdiv((uint32_t)k, g.dm, g.ds1, g.ds2);
+        const int off = off0 + (k - dy * g.kwC), ih = ih0 + dy;
+        float x = 0.0f;
+        if (k < g.K && ih >= 0 && ih < g.H && off >= 0 && off < g.WC) x = __ldg(img + (int64_t)ih * g.WC + off);
+        v[j] = x;
       }
-      v[j] = x;
     }
-  }
-  if (BF16) {
-    uint32_t o[4];
+    if (BF16) {
+      uint32_t o[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-      o[j] = *reinterpret_cast<uint32_t*>(&h);
-    }
-    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(q) + row * ldq + k0) = make_uint4(o[0], o[1], o[2], o[3]);
-  } else {
-    uint32_t lo = 0, hi = 0;
+      for (int j = 0; j < 4; ++j) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        o[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(q) + row * ldq + k0) = make_uint4(o[0], o[1], o[2], o[3]);
+    } else {
+      uint32_t lo = 0, hi = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      lo |= (uint32_t)(conv_code(v[j], inv_scale, qmax) & 0xff) << (8 * j);
-      hi |= (uint32_t)(conv_code(v[j + 4], inv_scale, qmax) & 0xff) << (8 * j);
+      for (int j = 0; j < 4; ++j) {
+        lo |= (uint32_t)(conv_code(v[j], inv_scale, qmax) & 0xff) << (8 * j);
+        hi |= (uint32_t)(conv_code(v[j + 4], inv_scale, qmax) & 0xff) << (8 * j);
+      }
+      *reinterpret_cast<uint2*>(reinterpret_cast<int8_t*>(q) + row * ldq + k0) = make_uint2(lo, hi);
     }
-    *reinterpret_cast<uint2*>(reinterpret_cast<int8_t*>(q) + row * ldq + k0) = make_uint2(lo, hi);
   }
 }
 
@@ -156,14 +175,21 @@ int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, 
   g.OH = (H + 2 * pad - kh) / stride + 1;
   g.OW = (W + 2 * pad - kw) / stride + 1;
   g.K = kh * kw * C;
+  g.kwC = kw * C; g.WC = W * C;
+  fastdiv_init((uint32_t)g.kwC, &g.dm, &g.ds1, &g.ds2);
   const int64_t rows = B * g.OH * g.OW;
   if (rows == 0) return QCFG_OK;
+  if (B * g.OH > 0x7fffffff || (int64_t)W * C > 0x7fffffff) return set_error(ctx, QCFG_ESHAPE, "im2col: image too large");
   const int vec = (C % 8 == 0 && (uintptr_t)src % 16 == 0) ? 1 : 0;
-  const int64_t total = rows * (ldq >> 3);
-  const unsigned blocks = (unsigned)((total + 255) / 256);
+  const int gpr = (int)(ldq >> 3);
+  const int bx = gpr >= 24 ? 32 : (gpr >= 12 ? 16 : 8);
+  const int by = 256 / bx;
+  const dim3 block((unsigned)bx, (unsigned)by);
+  const dim3 grid((unsigned)(B * g.OH), (unsigned)((g.OW + by - 1) / by));
+  if (grid.y > 65535) return set_error(ctx, QCFG_ESHAPE, "im2col: output row too wide");
   prof_begin(ctx, 2, st);
-  if (bits == 16) im2col_quantize_kernel<true><<<blocks, 256, 0, st>>>(src, rows, g, 1.0f, 0.0f, q, ldq, vec);
-  else im2col_quantize_kernel<false><<<blocks, 256, 0, st>>>(src, rows, g, inv_scale, qmax_of(bits), q, ldq, vec);
+  if (bits == 16) im2col_quantize_kernel<true><<<grid, block, 0, st>>>(src, g, 1.0f, 0.0f, q, ldq, vec);
+  else im2col_quantize_kernel<false><<<grid, block, 0, st>>>(src, g, inv_scale, qmax_of(bits), q, ldq, vec);
   prof_end(ctx, 2, 0.0, st);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "im2col launch");
