@@ -90,6 +90,10 @@ int qcfg_set_fusion(qcfg_ctx* ctx, int enabled);
  * outputs wider than 128 columns and more than 128 rows).  Off: every tile is 128 rows on one
  * CTA.  Results are bit-identical either way.                                               */
 int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled);
+/* Switches grouped launches in model evaluations (default on): up to three layers that do not
+ * depend on one another and share rows, reduction length, operand type and tile width run as
+ * one kernel.  Results are bit-identical either way.                                        */
+int qcfg_set_grouping(qcfg_ctx* ctx, int enabled);
 
 /* Per-launch timing of the GEMM kernel with CUDA events recorded on the launching stream
  * (off by default; a few microseconds of host time per launch when on).  kernel_class 0 is

@@ -21,6 +21,7 @@ struct Ctx {
   int64_t launches = 0;
   int fuse = 1;
   int pair = 1;                     // two-CTA GEMM tiles where they apply
+  int group = 1;                    // independent GEMMs of equal shape share a launch
   int pair_clusters[2] = {0, 0};
   char msg[512] = {0};
   // last sweep tables uploaded to the scratch buffer
@@ -242,10 +243,24 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     S.a_ready = false; S.a_ptr = nullptr; S.y_ptr = nullptr; S.pre_ptr = nullptr;
     S.bits = calibrate ? 16 : bits[l];
   }
+  // GEMMs that are ready together and have the same m, k, operand type and tile width (the three
+  // projections of an attention block) are collected and launched as one grouped kernel.
+  std::vector<GemmArgs> pending;
+  std::vector<int> pending_layers;
+  auto flush = [&]() -> int {
+    if (pending.empty()) return QCFG_OK;
+    const int frc = launch_gemm_group(ctx, pending.data(), (int)pending.size(), st);
+    pending.clear();
+    pending_layers.clear();
+    return frc;
+  };
+  const bool grouping = ctx->group && !layer_ev;
   for (int l = 0; l < n; ++l) {
     LayerState& S = M->L[l];
     const qcfg_layer& d = S.d;
     const int b = S.bits;
+    for (int pl : pending_layers)
+      if (d.src == pl || d.residual_from == pl) { const int frc = flush(); if (frc) return frc; break; }
     int rc = ensure_weight_codes(ctx, S, b, st);
     if (rc) return rc;
     // optional per-layer timing: everything this layer launches (operand preparation and GEMM)
@@ -380,11 +395,17 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       if (!R.y_ptr || R.rows != S.rows) return set_error(ctx, QCFG_ESHAPE, "layer %d: shortcut from layer %d is unavailable or has other rows", l, d.residual_from);
       g.residual = R.y_ptr; g.ldr = R.d.n_out;
     }
-    rc = launch_gemm(ctx, g, st);
-    if (rc) return rc;
+    if (grouping) {
+      if (!pending.empty() && (pending.size() == 3 || !gemm_groupable(pending[0], g))) { rc = flush(); if (rc) return rc; }
+      pending.push_back(g);
+      pending_layers.push_back(l);
+    } else {
+      rc = launch_gemm(ctx, g, st);
+      if (rc) return rc;
+    }
     if (layer_ev && cudaEventRecord(layer_ev[2 * l + 1], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
   }
-  return QCFG_OK;
+  return flush();
 }
 
 }  // namespace
@@ -474,6 +495,11 @@ int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* laun
 int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled) {
   if (!ctx) return QCFG_EINVAL;
   ctx->c.pair = enabled ? 1 : 0;
+  return QCFG_OK;
+}
+int qcfg_set_grouping(qcfg_ctx* ctx, int enabled) {
+  if (!ctx) return QCFG_EINVAL;
+  ctx->c.group = enabled ? 1 : 0;
   return QCFG_OK;
 }
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled) {

@@ -84,6 +84,9 @@ struct GemmArgs {
   CodeSlot slots[kMaxSlots];
 };
 int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st);
+// up to three GEMMs of equal m, k, operand type and tile width in one launch
+bool gemm_groupable(const GemmArgs& a, const GemmArgs& b);
+int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st);
 int gemm_init(Ctx* ctx);   // resolves the tensor-map encoder, sets smem attributes
 
 // ----- small device helpers -----------------------------------------------------------

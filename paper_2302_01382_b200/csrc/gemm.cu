@@ -46,18 +46,27 @@ struct OutDesc {
   int64_t ld;         // elements
   float inv_scale, qmax;
 };
-struct OutMaps { CUtensorMap m[kNumOuts]; };
-
-struct GemmParams {
-  int32_t m, n, k_blocks, bn, tiles_m, tiles_n, stages, is_bf16;
-  int32_t epi_bytes;          // staging bytes per epilogue warp (2048 or 4096)
-  uint32_t idesc;
+// One launch runs up to kMaxGroups GEMMs of equal m, k, operand type and tile shape ("groups":
+// layers that are ready at the same time, e.g. the three projections reading one input).  Their
+// column tiles are numbered one after the other, so the persistent CTAs work through all of them
+// and only the first tile's main loop and the last tile's epilogue stay unoverlapped.
+constexpr int kMaxGroups = 3;
+struct GroupMaps { CUtensorMap a, b, om[kNumOuts]; };
+struct AllMaps { GroupMaps g[kMaxGroups]; };
+struct GroupDesc {
+  int32_t n, tn_begin;        // columns; first column-tile index of the group in the launch's numbering
+  int32_t act;
+  int32_t need_y;             // anything besides raw accumulators to produce
   float scale_x;
   const float* scale_w;
-  int32_t act;
   const float* residual; int64_t ldr;
-  int32_t need_y;             // anything besides raw accumulators to produce
   OutDesc outs[kNumOuts];     // [0] raw accumulators, [1] fp32 output, [2..] consumer codes
+};
+struct GemmParams {
+  int32_t m, k_blocks, bn, tiles_m, tiles_n, stages, is_bf16;   // tiles_n: column tiles of all groups together
+  int32_t epi_bytes;          // staging bytes per epilogue warp (2048 or 4096)
+  uint32_t idesc;
+  GroupDesc grp[kMaxGroups];  // unused groups have tn_begin = INT32_MAX
   unsigned* err;
 };
 
@@ -324,14 +333,15 @@ __device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap*
 
 // One 32-column chunk of one accumulator row (all 32 lanes of the warp call this together).
 template <bool BF16>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMaps& om, uint32_t (&v)[32], float cs_lane,
+__device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtensorMap* om, int m, uint32_t epi_bytes,
+                                               uint32_t (&v)[32], float cs_lane,
                                                int64_t row, int row0, int col0, uint32_t stage, uint32_t& cursor, int lane) {
   const int ncols = p.n - col0;                    // valid columns in this chunk (may be <= 0 or > 32)
-  if (ncols <= 0 || row0 >= p.m) return;           // warp-uniform: the piece lies outside the matrix
-  const bool row_ok = row < p.m;
+  if (ncols <= 0 || row0 >= m) return;             // warp-uniform: the piece lies outside the matrix
+  const bool row_ok = row < m;
   const bool full = ncols >= 32;
 
-  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &om.m[0], v, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
+  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &om[0], v, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
   if (!p.need_y) return;
 
   float y[32];
@@ -371,7 +381,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
     uint32_t w[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(y[i]);
-    store_piece<32>(p.outs[1], &om.m[1], w, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
+    store_piece<32>(p.outs[1], &om[1], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
   }
 #pragma unroll
   for (int s = 0; s < kMaxSlots; ++s) {
@@ -382,7 +392,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
       for (int i = 0; i < 8; ++i)
         w[i] = pack4(code_word(y[4 * i], o.inv_scale, o.qmax), code_word(y[4 * i + 1], o.inv_scale, o.qmax),
                      code_word(y[4 * i + 2], o.inv_scale, o.qmax), code_word(y[4 * i + 3], o.inv_scale, o.qmax));
-      store_piece<8>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
+      store_piece<8>(o, &om[2 + s], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
     } else if (o.kind == 2) {
       uint32_t w[16];
 #pragma unroll
@@ -390,17 +400,16 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const OutMap
         __nv_bfloat162 h = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
         w[i] = *reinterpret_cast<uint32_t*>(&h);
       }
-      store_piece<16>(o, &om.m[2 + s], w, row_ok, ncols, row, row0, col0, stage, (uint32_t)p.epi_bytes, cursor, lane);
+      store_piece<16>(o, &om[2 + s], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
     }
   }
 }
 
 // ---------------------------------------------------------------------------- the kernel
 
-template <bool BF16, bool PAIR>
+template <bool BF16, bool PAIR, bool GROUPED>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ OutMaps omaps, const __grid_constant__ GemmParams p) {
+gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the 128B swizzle atoms
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -425,6 +434,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // first tile of this CTA (pair)
   const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int rows_per_tile = PAIR ? 2 * BM : BM;
+  // group of a column tile (a single-GEMM launch has only group 0, known at compile time)
+  auto group_of = [&](int tn) -> int {
+    return GROUPED ? (int)(tn >= p.grp[1].tn_begin) + (int)(tn >= p.grp[2].tn_begin) : 0;
+  };
   // Tiles are numbered with the row-tile index fastest.  Each role walks its tiles by adding the
   // stride split into (row tiles, column tiles) once here: a division per tile would sit on the
   // epilogue's and the producer's path.
@@ -443,9 +456,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   uint32_t ld_dst = stage0, ld_bar = full0;      // stage address and its full barrier
   int ld_x = 0, ld_ya = 0, ld_yb = 0;            // TMA coordinates of the next k-block
   int ld_tm = tm0, ld_tn = tn0;
+  const CUtensorMap* ld_map_a = &maps.g[0].a;
+  const CUtensorMap* ld_map_b = &maps.g[0].b;
   auto set_tile_coords = [&]() {
+    const int g = group_of(ld_tn);
+    if (GROUPED) { ld_map_a = &maps.g[g].a; ld_map_b = &maps.g[g].b; }
     ld_ya = ld_tm * rows_per_tile + rank * BM;
-    ld_yb = ld_tn * p.bn + rank * b_rows;
+    ld_yb = (ld_tn - (GROUPED ? p.grp[g].tn_begin : 0)) * p.bn + rank * b_rows;
   };
   set_tile_coords();
   const bool elected = elect_one();    // the lane of a converged warp that issues TMA / MMA instructions
@@ -454,12 +471,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (PAIR) {
       // the first CTA's barrier collects the bytes of both CTAs' loads
       if (rank == 0) mbar_expect_tx(ld_bar, 2 * stage_bytes);
-      tma_load_2d_pair(ld_dst, &map_a, ld_bar, ld_x, ld_ya);
-      tma_load_2d_pair(ld_dst + BM * kStageKBytes, &map_b, ld_bar, ld_x, ld_yb);
+      tma_load_2d_pair(ld_dst, ld_map_a, ld_bar, ld_x, ld_ya);
+      tma_load_2d_pair(ld_dst + BM * kStageKBytes, ld_map_b, ld_bar, ld_x, ld_yb);
     } else {
       mbar_expect_tx(ld_bar, stage_bytes);
-      tma_load_2d(ld_dst, &map_a, ld_bar, ld_x, ld_ya);
-      tma_load_2d(ld_dst + BM * kStageKBytes, &map_b, ld_bar, ld_x, ld_yb);
+      tma_load_2d(ld_dst, ld_map_a, ld_bar, ld_x, ld_ya);
+      tma_load_2d(ld_dst + BM * kStageKBytes, ld_map_b, ld_bar, ld_x, ld_yb);
     }
     }
     ld_dst += stage_bytes; ld_bar += 8; ld_x += k_elems;
@@ -473,8 +490,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   };
 
   if (threadIdx.x == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.g[0].a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.g[0].b) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
     *abort_flag = 0;
@@ -586,12 +603,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // the top of the loop, and a load issued there would put its whole latency on the tile.
     auto load_scales = [&](int tile, int tile_tn, float (&w)[2]) {
       w[0] = 0.f; w[1] = 0.f;
-      if (BF16 || !p.need_y || tile >= num_tiles) return;
-      const int cb = tile_tn * p.bn + c_begin * 32;
+      if (BF16 || tile >= num_tiles) return;
+      const GroupDesc& G = p.grp[group_of(tile_tn)];
+      if (!G.need_y) return;
+      const int cb = (tile_tn - (GROUPED ? G.tn_begin : 0)) * p.bn + c_begin * 32;
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int col = cb + j * 32 + lane;
-        if (c_begin + j < c_end && col < p.n) w[j] = __ldg(p.scale_w + col);
+        if (c_begin + j < c_end && col < G.n) w[j] = __ldg(G.scale_w + col);
       }
     };
     float sw_next[2];
@@ -600,8 +619,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
       const int a = t & 1;
       const int row0 = tm * rows_per_tile + rank * BM + quad * 32;
-      const int col_base = tn * p.bn + c_begin * 32;
-      const float cs[2] = {__fmul_rn(p.scale_x, sw_next[0]), __fmul_rn(p.scale_x, sw_next[1])};
+      const int g = group_of(tn);
+      const GroupDesc& G = p.grp[g];
+      const int col_base = (tn - (GROUPED ? G.tn_begin : 0)) * p.bn + c_begin * 32;
+      const float cs[2] = {__fmul_rn(G.scale_x, sw_next[0]), __fmul_rn(G.scale_x, sw_next[1])};
       int tm_next = tm + step_tm, tn_next = tn + step_tn;
       if (tm_next >= p.tiles_m) { tm_next -= p.tiles_m; ++tn_next; }
       load_scales(tile + tile_step, tn_next, sw_next);
@@ -621,7 +642,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           __syncwarp();
           if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
         }
-        epilogue_chunk<BF16>(p, omaps, v, c ? cs[1] : cs[0], row, row0, col_base + 32 * c, stage, cursor, lane);
+        epilogue_chunk<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, c ? cs[1] : cs[0], row, row0, col_base + 32 * c, stage, cursor, lane);
       }
       if (nch == 0) {
         __syncwarp();
@@ -696,76 +717,101 @@ int gemm_init(Ctx* ctx) {
       return set_error(ctx, QCFG_ECUDA, "cuTensorMapEncodeTiled entry point not found");
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+  cudaError_t e = cudaSuccess;
+  const void* kernels[8] = {
+      (const void*)gemm_kernel<false, false, false>, (const void*)gemm_kernel<false, false, true>,
+      (const void*)gemm_kernel<false, true, false>,  (const void*)gemm_kernel<false, true, true>,
+      (const void*)gemm_kernel<true, false, false>,  (const void*)gemm_kernel<true, false, true>,
+      (const void*)gemm_kernel<true, true, false>,   (const void*)gemm_kernel<true, true, true>};
+  for (int i = 0; i < 8 && e == cudaSuccess; ++i)
+    e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
   return check_cuda(ctx, e, "gemm smem attribute");
 }
 
-int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
-  if (g.m <= 0 || g.n <= 0 || g.k <= 0) return set_error(ctx, QCFG_ESHAPE, "gemm: m, n, k must be positive");
-  const int esz = g.is_bf16 ? 2 : 1;
-  if (((uintptr_t)g.a & 15) || ((uintptr_t)g.b & 15) || (g.lda * esz) % 16 || (g.ldb * esz) % 16)
-    return set_error(ctx, QCFG_EALIGN, "gemm: operands need 16-byte aligned pointers and row strides");
-  if (g.lda < g.k || g.ldb < g.k) return set_error(ctx, QCFG_ESHAPE, "gemm: leading dimension below k");
-  if (g.m > 0x7fffffff || g.n > 0x7fffffff) return set_error(ctx, QCFG_ESHAPE, "gemm: dimension too large");
+// Tile width a GEMM of n columns gets.
+static int tile_n_of(int64_t n) { return n <= 32 ? 32 : n <= 64 ? 64 : n <= 128 ? 128 : 256; }
+
+bool gemm_groupable(const GemmArgs& a, const GemmArgs& b) {
+  return a.m == b.m && a.k == b.k && a.is_bf16 == b.is_bf16 && tile_n_of(a.n) == tile_n_of(b.n);
+}
+
+int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) {
+  if (count < 1 || count > kMaxGroups) return set_error(ctx, QCFG_EINVAL, "gemm: %d groups", count);
+  const GemmArgs& g0 = gs[0];
+  const int esz = g0.is_bf16 ? 2 : 1;
+  const int bn = tile_n_of(g0.n);
+  for (int i = 0; i < count; ++i) {
+    const GemmArgs& g = gs[i];
+    if (g.m <= 0 || g.n <= 0 || g.k <= 0) return set_error(ctx, QCFG_ESHAPE, "gemm: m, n, k must be positive");
+    if (((uintptr_t)g.a & 15) || ((uintptr_t)g.b & 15) || (g.lda * esz) % 16 || (g.ldb * esz) % 16)
+      return set_error(ctx, QCFG_EALIGN, "gemm: operands need 16-byte aligned pointers and row strides");
+    if (g.lda < g.k || g.ldb < g.k) return set_error(ctx, QCFG_ESHAPE, "gemm: leading dimension below k");
+    if (g.m > 0x7fffffff || g.n > 0x7fffffff) return set_error(ctx, QCFG_ESHAPE, "gemm: dimension too large");
+    if (i && !gemm_groupable(g0, g)) return set_error(ctx, QCFG_EINVAL, "gemm: grouped launches need equal m, k, type and tile width");
+  }
 
   GemmParams p{};
-  p.m = (int32_t)g.m; p.n = (int32_t)g.n;
-  const int64_t kbytes = g.k * esz;
+  p.m = (int32_t)g0.m;
+  const int64_t kbytes = g0.k * esz;
   p.k_blocks = (int32_t)((kbytes + kStageKBytes - 1) / kStageKBytes);
-  int bn = 256;
-  if (g.n <= 32) bn = 32; else if (g.n <= 64) bn = 64; else if (g.n <= 128) bn = 128;
   p.bn = bn;
   // pair flavour (two CTAs per 256-row tile, cta_group::2) for wide outputs with at least two
-  // row tiles: it halves the B bytes each SM pulls from L2, which is what limits the main loop
-  const bool pair = ctx_pair_enabled(ctx) && bn == 256 && g.m > BM && sm_count(ctx) >= 2;
+  // row tiles: it halves the B bytes each SM stages per k-block
+  const bool pair = ctx_pair_enabled(ctx) && bn == 256 && g0.m > BM && sm_count(ctx) >= 2;
   const int tile_rows = pair ? 2 * BM : BM;
-  p.tiles_m = (int32_t)((g.m + tile_rows - 1) / tile_rows);
-  p.tiles_n = (int32_t)((g.n + bn - 1) / bn);
+  p.tiles_m = (int32_t)((g0.m + tile_rows - 1) / tile_rows);
   const int stage_bytes = (BM + (pair ? bn / 2 : bn)) * kStageKBytes;
-  p.is_bf16 = g.is_bf16;
+  p.is_bf16 = g0.is_bf16;
   // instruction descriptor: D format (F32 = 1, S32 = 2) at bit 4, A/B format (BF16 = 1, S8 = 1)
   // at bits 7 and 10, both operands K-major, N/8 at bit 17, M/16 at bit 24
-  p.idesc = ((g.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(tile_rows >> 4) << 24);
-  p.scale_x = g.scale_x; p.scale_w = g.scale_w; p.act = g.act;
-  p.residual = g.residual; p.ldr = g.ldr;
-  if (g.acc && !g.is_bf16) { p.outs[0].kind = 4; p.outs[0].ptr = g.acc; p.outs[0].ld = g.n; }
-  if (g.y) { p.outs[1].kind = 3; p.outs[1].ptr = g.y; p.outs[1].ld = g.ldy; }
-  p.need_y = g.y != nullptr;
-  for (int s = 0; s < kMaxSlots; ++s) {
-    if (!g.slots[s].kind) continue;
-    OutDesc& o = p.outs[2 + s];
-    o.kind = g.slots[s].kind; o.ptr = g.slots[s].ptr; o.ld = g.slots[s].ld;
-    o.inv_scale = g.slots[s].inv_scale; o.qmax = g.slots[s].qmax;
-    p.need_y = 1;
-  }
-  if (!p.need_y && !p.outs[0].kind) return set_error(ctx, QCFG_EINVAL, "gemm: no output requested");
-  if (p.need_y && !g.is_bf16 && !g.scale_w) return set_error(ctx, QCFG_EINVAL, "gemm: scale_w is null");
+  p.idesc = ((g0.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(tile_rows >> 4) << 24);
   p.err = err_word(ctx);
-  OutMaps om;
-  memset(&om, 0, sizeof(om));
-  for (int i = 0; i < kNumOuts; ++i)
-    if (p.outs[i].kind) p.outs[i].tma = make_out_map(&om.m[i], p.outs[i], g.m, g.n) ? 1 : 0;
 
-  // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
+  AllMaps maps;
+  memset(&maps, 0, sizeof(maps));
   bool wide = false;
-  for (int i = 0; i < kNumOuts; ++i) if (p.outs[i].kind >= 2 && p.outs[i].tma) wide = true;
+  int32_t tn_total = 0;
+  double ops = 0.0;
+  for (int i = 0; i < kMaxGroups; ++i) p.grp[i].tn_begin = 0x7fffffff;
+  for (int i = 0; i < count; ++i) {
+    const GemmArgs& g = gs[i];
+    GroupDesc& G = p.grp[i];
+    G.n = (int32_t)g.n;
+    G.tn_begin = tn_total;
+    tn_total += (int32_t)((g.n + bn - 1) / bn);
+    G.scale_x = g.scale_x; G.scale_w = g.scale_w; G.act = g.act;
+    G.residual = g.residual; G.ldr = g.ldr;
+    if (g.acc && !g.is_bf16) { G.outs[0].kind = 4; G.outs[0].ptr = g.acc; G.outs[0].ld = g.n; }
+    if (g.y) { G.outs[1].kind = 3; G.outs[1].ptr = g.y; G.outs[1].ld = g.ldy; }
+    G.need_y = g.y != nullptr;
+    for (int s = 0; s < kMaxSlots; ++s) {
+      if (!g.slots[s].kind) continue;
+      OutDesc& o = G.outs[2 + s];
+      o.kind = g.slots[s].kind; o.ptr = g.slots[s].ptr; o.ld = g.slots[s].ld;
+      o.inv_scale = g.slots[s].inv_scale; o.qmax = g.slots[s].qmax;
+      G.need_y = 1;
+    }
+    if (!G.need_y && !G.outs[0].kind) return set_error(ctx, QCFG_EINVAL, "gemm: no output requested");
+    if (G.need_y && !g.is_bf16 && !g.scale_w) return set_error(ctx, QCFG_EINVAL, "gemm: scale_w is null");
+    for (int j = 0; j < kNumOuts; ++j)
+      if (G.outs[j].kind) G.outs[j].tma = make_out_map(&maps.g[i].om[j], G.outs[j], g.m, g.n) ? 1 : 0;
+    // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
+    for (int j = 0; j < kNumOuts; ++j) if (G.outs[j].kind >= 2 && G.outs[j].tma) wide = true;
+    int rc = make_map(ctx, &maps.g[i].a, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
+    if (rc == QCFG_OK) rc = make_map(ctx, &maps.g[i].b, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
+    if (rc != QCFG_OK) return rc;
+    ops += 2.0 * (double)g.m * (double)g.n * (double)g.k;
+  }
+  p.tiles_n = tn_total;
   p.epi_bytes = wide ? 4096 : 2048;
   int stages = (kSmemMax - kSmemHeader - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   p.stages = stages;
 
-  CUtensorMap ma, mb;
-  int rc = make_map(ctx, &ma, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
-  if (rc == QCFG_OK) rc = make_map(ctx, &mb, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
-  if (rc != QCFG_OK) return rc;
-
   const int num_tiles = p.tiles_m * p.tiles_n;
   int grid = sm_count(ctx);
   if (pair) {
-    int* cached = pair_cluster_cache(ctx) + (g.is_bf16 ? 1 : 0);
+    int* cached = pair_cluster_cache(ctx) + (g0.is_bf16 ? 1 : 0);
     if (*cached == 0) {     // how many CTA pairs the device keeps resident at once
       cudaLaunchConfig_t q = {};
       q.gridDim = dim3((unsigned)(grid & ~1));
@@ -776,8 +822,8 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
       qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
       q.attrs = qa; q.numAttrs = 1;
       int n = 0;
-      cudaError_t oe = g.is_bf16 ? cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true, true>, &q)
-                                 : cudaOccupancyMaxActiveClusters(&n, gemm_kernel<false, true>, &q);
+      cudaError_t oe = g0.is_bf16 ? cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true, true, false>, &q)
+                                  : cudaOccupancyMaxActiveClusters(&n, gemm_kernel<false, true, false>, &q);
       if (oe != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = grid / 2; }
       if (n > grid / 2) n = grid / 2;
       *cached = n;
@@ -801,16 +847,19 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 2 : 1;
-  prof_begin(ctx, g.is_bf16 ? 1 : 0, st);
-  cudaError_t le;
-  if (pair) le = g.is_bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, true>, ma, mb, om, p)
-                           : cudaLaunchKernelEx(&cfg, gemm_kernel<false, true>, ma, mb, om, p);
-  else le = g.is_bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, false>, ma, mb, om, p)
-                      : cudaLaunchKernelEx(&cfg, gemm_kernel<false, false>, ma, mb, om, p);
-  prof_end(ctx, g.is_bf16 ? 1 : 0, 2.0 * (double)g.m * (double)g.n * (double)g.k, st);
+  using Kern = void (*)(const AllMaps, const GemmParams);
+  static const Kern kernels[8] = {
+      gemm_kernel<false, false, false>, gemm_kernel<false, false, true>, gemm_kernel<false, true, false>, gemm_kernel<false, true, true>,
+      gemm_kernel<true, false, false>,  gemm_kernel<true, false, true>,  gemm_kernel<true, true, false>,  gemm_kernel<true, true, true>};
+  const Kern kern = kernels[(g0.is_bf16 ? 4 : 0) + (pair ? 2 : 0) + (count > 1 ? 1 : 0)];
+  prof_begin(ctx, g0.is_bf16 ? 1 : 0, st);
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, maps, p);
+  prof_end(ctx, g0.is_bf16 ? 1 : 0, ops, st);
   if (le != cudaSuccess) return check_cuda(ctx, le, "gemm launch");
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "gemm launch");
 }
+
+int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st) { return launch_gemm_group(ctx, &g, 1, st); }
 
 }  // namespace qcfg

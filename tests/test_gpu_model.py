@@ -151,6 +151,31 @@ def test_fused_and_unfused_agree_bitwise_and_taps_are_optional(ctx):
     model.close()
 
 
+@pytest.mark.parametrize("bits_kind", ["uniform8", "mixed_int", "with16"])
+def test_grouped_and_single_launches_agree_bitwise(ctx, bits_kind):
+    """The three projections of a block read one input: when their GEMMs have the same shape and
+    operand type they run as one grouped launch (also with different bit widths, i.e. different
+    input codes and scales per group); a 16-bit layer among them splits the group."""
+    w = wl.bert_stack(23, 700, 256, 1024, 2, bit_choices=(4, 8))
+    n = len(w.layers)
+    bits = {"uniform8": [8] * n, "mixed_int": [4, 8, 6, 8, 3, 8] * 2, "with16": [8, 16, 8, 4, 16, 8] * 2}[bits_kind]
+    model, x = build(ctx, w)
+    res = []
+    for grouping in (True, False):
+        ctx.set_grouping(grouping)
+        try:
+            ys = run_eval(ctx, model, w, x, bits)
+        finally:
+            ctx.set_grouping(True)
+        res.append(ys)
+    for a, b in zip(*res):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    act_g = np.array(model.act_absmax(), np.float32)
+    w_amax = [np.array(model.weight_absmax(l), np.float32) for l in range(n)]
+    teacher_forced_check(ctx, model, w, x, bits, res[0], act_g, w_amax)
+    model.close()
+
+
 def test_model_argument_errors(ctx):
     import paper_2302_01382_b200 as q
     w = wl.tiny_mlp()
