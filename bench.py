@@ -37,7 +37,7 @@ TOKENS = 32 * 384
 WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
 # DRAM bytes (read + write) per int8 GEMM launch from the ncu capture summarised in
 # profiles/gemm_int8_bert_base_block.md; set to None whenever the GEMM kernel changes.
-GEMM_TRAFFIC_BYTES = 16.2e6
+GEMM_TRAFFIC_BYTES = None
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -334,6 +334,8 @@ def run_gpu(args):
     search = None
     if not args.no_e2e:
         rank_now = [int(v) for v in job.last_ranking]
+        job.model.search(q.SEARCH_GREEDY, rank_now, [8, 4], 0.9, job.x, w.m)     # untimed: allocates the driver's buffers
+        torch.cuda.synchronize()
         t0 = time.perf_counter()
         bits_s, vis_s, acc_s, n_s = job.model.search(q.SEARCH_GREEDY, rank_now, [8, 4], 0.9, job.x, w.m)
         torch.cuda.synchronize()
