@@ -37,7 +37,7 @@ TOKENS = 32 * 384
 WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
 # DRAM bytes (read + write) per int8 GEMM launch from the ncu capture summarised in
 # profiles/gemm_int8_bert_base_block.md; set to None whenever the GEMM kernel changes.
-GEMM_TRAFFIC_BYTES = None
+GEMM_TRAFFIC_BYTES = 27.4e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -359,7 +359,7 @@ def run_gpu(args):
                          "unit": "TOP/s", "frac": achieved / int8_peak,
                          "peak_source": f"2 x sustained bf16 cuBLAS ({peaks['_source']})",
                          "launches": int(g_n), "avg_launch_us": 1e3 * g_ms / max(g_n, 1), "traffic": GEMM_TRAFFIC_BYTES,
-                         "traffic_source": "ncu dram bytes per launch, mean of the six GEMMs of one block at 12288 tokens",
+                         "traffic_source": "ncu dram bytes per launch, mean of the four GEMM launches (q/k/v grouped, o, ffn1, ffn2) of one block at 12288 tokens",
                          "share_of_kernel_time": g_ms / max(g_ms + b_ms + o_ms, 1e-9), "share_of_step": g_ms / instrumented_ms,
                          "how": "CUDA events around every launch in a second pass over the same steps"},
             "sweep": {"gbs": sweep_gbs, "ms": sweep_ms, "bytes": sweep_bytes, "hbm_peak_gbs": peaks["hbm_gbs"],
