@@ -6,6 +6,9 @@ added to tensor w_i alone.  Readings: the second argument of N is the standard d
 is the whole tensor's maximum; the loss (the paper's needs labels) is the relative L2 distance of
 the last layer's output from the noise-free output, so L(x, W) = 0; the model is the 16-bit
 floating-point baseline.  The standard-normal draws are inputs.
+
+Parity unpinned: the loss.  The paper's L needs labels; the output-distance proxy used here is this
+build's convention, so no value in the paper can pin it (the arithmetic around it is pinned).
 """
 import numpy as np
 
