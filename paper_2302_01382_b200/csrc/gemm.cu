@@ -53,10 +53,14 @@ struct OutDesc {
 constexpr int kMaxGroups = 3;
 struct GroupMaps { CUtensorMap a, b, om[kNumOuts]; };
 struct AllMaps { GroupMaps g[kMaxGroups]; };
+// Epilogue bodies.  The general one handles any combination of outputs with run-time branches; the
+// two common combinations have straight-line bodies (same arithmetic, same order).
+enum : int32_t { EPI_GENERAL = 0, EPI_CODES1 = 1, EPI_Y = 2 };
 struct GroupDesc {
   int32_t n, tn_begin;        // columns; first column-tile index of the group in the launch's numbering
   int32_t act;
   int32_t need_y;             // anything besides raw accumulators to produce
+  int32_t mode;               // EPI_*: which epilogue body serves this group
   float scale_x;
   const float* scale_w;
   const float* residual; int64_t ldr;
@@ -328,6 +332,79 @@ __device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap*
         else dst[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
       }
     }
+  }
+}
+
+// Rescale (and activate) one chunk: y[i] = act(acc[i] * cs[col i]); lane i holds the scale of column i.
+template <bool BF16>
+__device__ __forceinline__ void chunk_values(float (&y)[32], const uint32_t (&v)[32], float cs_lane, int act) {
+  if (BF16) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      y[i] = __fmul_rn((float)(int32_t)v[i], __shfl_sync(0xffffffffu, cs_lane, i));
+  }
+  if (act == QCFG_ACT_RELU) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = fmaxf(y[i], 0.0f);
+  } else if (act == QCFG_ACT_GELU_TANH) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = gelu_tanh(y[i]);
+  }
+}
+
+// EPI_CODES1: the only output is one int8 code matrix (slot 0) written by TMA; no shortcut.
+template <bool BF16>
+__device__ __forceinline__ void epilogue_chunk_codes1(const GroupDesc& p, const CUtensorMap* om, int m, uint32_t epi_bytes,
+                                                      const uint32_t (&v)[32], float cs_lane, int row0, int col0,
+                                                      uint32_t stage, uint32_t& cursor, int lane) {
+  if (p.n - col0 <= 0 || row0 >= m) return;        // warp-uniform: the piece lies outside the matrix
+  float y[32];
+  chunk_values<BF16>(y, v, cs_lane, p.act);
+  const float inv = p.outs[2].inv_scale, qmax = p.outs[2].qmax;
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    w[i] = pack4(code_word(y[4 * i], inv, qmax), code_word(y[4 * i + 1], inv, qmax),
+                 code_word(y[4 * i + 2], inv, qmax), code_word(y[4 * i + 3], inv, qmax));
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+  __syncwarp();
+  const uint32_t base = stage + (cursor & 1u) * (epi_bytes >> 1);
+  ++cursor;
+  st_shared_v4(base + lane * 32, w[0], w[1], w[2], w[3]);
+  st_shared_v4(base + lane * 32 + 16, w[4], w[5], w[6], w[7]);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) tma_store_2d(&om[2], base, col0, row0);
+}
+
+// EPI_Y: the only output is the fp32 matrix written by TMA (two 16-column pieces); no shortcut.
+template <bool BF16>
+__device__ __forceinline__ void epilogue_chunk_y(const GroupDesc& p, const CUtensorMap* om, int m, uint32_t epi_bytes,
+                                                 const uint32_t (&v)[32], float cs_lane, int row0, int col0,
+                                                 uint32_t stage, uint32_t& cursor, int lane) {
+  const int ncols = p.n - col0;
+  if (ncols <= 0 || row0 >= m) return;
+  float y[32];
+  chunk_values<BF16>(y, v, cs_lane, p.act);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    if (h == 1 && ncols <= 16) break;
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    __syncwarp();
+    const uint32_t base = stage + (cursor & 1u) * (epi_bytes >> 1);
+    ++cursor;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int js = j ^ ((lane >> 1) & 3);
+      st_shared_v4(base + lane * 64 + js * 16, __float_as_uint(y[16 * h + 4 * j]), __float_as_uint(y[16 * h + 4 * j + 1]),
+                   __float_as_uint(y[16 * h + 4 * j + 2]), __float_as_uint(y[16 * h + 4 * j + 3]));
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) tma_store_2d(&om[1], base, col0 + 16 * h, row0);
   }
 }
 
@@ -642,7 +719,13 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
           __syncwarp();
           if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
         }
-        epilogue_chunk<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, c ? cs[1] : cs[0], row, row0, col_base + 32 * c, stage, cursor, lane);
+        const float csl = c ? cs[1] : cs[0];
+        if (G.mode == EPI_CODES1)
+          epilogue_chunk_codes1<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row0, col_base + 32 * c, stage, cursor, lane);
+        else if (G.mode == EPI_Y)
+          epilogue_chunk_y<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row0, col_base + 32 * c, stage, cursor, lane);
+        else
+          epilogue_chunk<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
       }
       if (nch == 0) {
         __syncwarp();
@@ -797,6 +880,11 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       if (G.outs[j].kind) G.outs[j].tma = make_out_map(&maps.g[i].om[j], G.outs[j], g.m, g.n) ? 1 : 0;
     // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
     for (int j = 0; j < kNumOuts; ++j) if (G.outs[j].kind >= 2 && G.outs[j].tma) wide = true;
+    G.mode = EPI_GENERAL;
+    if (!G.residual && !G.outs[0].kind && !G.outs[3].kind && !G.outs[4].kind) {
+      if (!G.outs[1].kind && G.outs[2].kind == 1 && G.outs[2].tma) G.mode = EPI_CODES1;
+      else if (G.outs[1].kind && G.outs[1].tma && !G.outs[2].kind) G.mode = EPI_Y;
+    }
     int rc = make_map(ctx, &maps.g[i].a, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
     if (rc == QCFG_OK) rc = make_map(ctx, &maps.g[i].b, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
     if (rc != QCFG_OK) return rc;
