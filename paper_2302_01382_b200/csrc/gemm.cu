@@ -257,9 +257,11 @@ __device__ __forceinline__ float gelu_tanh(float y) {
 // int8 code of Eq. 1 in the low byte of the returned word: clamp, then add 1.5*2^23 (a
 // round-half-even at integer granularity); the low mantissa byte is the two's-complement code.
 __device__ __forceinline__ uint32_t code_word(float y, float inv_scale, float qmax) {
-  float t = __fmul_rn(y, inv_scale);
-  t = fminf(fmaxf(t, -qmax), qmax);
-  return __float_as_uint(__fadd_rn(t, 12582912.0f));
+  const float t = __fmul_rn(y, inv_scale);
+  // clamp to [-qmax, qmax] in one instruction: magnitude min(|t|, qmax), sign of t (qmax > 0)
+  float c;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c) : "f"(t), "f"(qmax));
+  return __float_as_uint(__fadd_rn(c, 12582912.0f));
 }
 // low bytes of four words -> one word (byte i from word i)
 __device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
