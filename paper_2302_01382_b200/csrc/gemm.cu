@@ -37,7 +37,6 @@ constexpr int kSmemMax = 232448;      // 227 KB
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 constexpr int kNumOuts = 2 + kMaxSlots;   // raw accumulators, fp32 output, consumer code slots
-constexpr int kEpiStageMax = 4096;        // per epilogue warp: one 32 x 128-byte piece, or two 1 KB code pieces
 
 struct OutDesc {
   int32_t kind;       // 0 none, 1 int8 codes, 2 bf16 codes, 3 fp32, 4 int32
