@@ -98,10 +98,17 @@ static void fastdiv_init(uint32_t d, uint32_t* m, uint32_t* s1, uint32_t* s2) {
   *s2 = l > 0 ? l - 1 : 0;
 }
 
-__device__ __forceinline__ int conv_code(float x, float inv_scale, float qmax) {
-  float t = __fmul_rn(x, inv_scale);
-  t = fminf(fmaxf(t, -qmax), qmax);
-  return __float2int_rn(t);
+// int8 code of Eq. 1 in the low byte of the returned word: one multiply, the clamp to +-qmax as
+// min(|t|, qmax) with t's sign, and a round-half-even by adding 1.5 * 2^23 (the low mantissa byte is
+// then the two's-complement code) -- all on the fp32 pipe, no float-to-int conversion.
+__device__ __forceinline__ uint32_t conv_code(float x, float inv_scale, float qmax) {
+  const float t = __fmul_rn(x, inv_scale);
+  float c;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c) : "f"(t), "f"(qmax));
+  return __float_as_uint(__fadd_rn(c, 12582912.0f));
+}
+__device__ __forceinline__ uint32_t conv_pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
 }
 
 // Operand row (b, oh, ow) holds the patch in (kh, kw, cin) order.  For a fixed kernel row dy the kw * C
@@ -137,6 +144,18 @@ __global__ void __launch_bounds__(256) im2col_quantize_kernel(const float* __res
 #pragma unroll
         for (int j = 0; j < 8; ++j) v[j] = 0.0f;
       }
+    } else if (g.kwC >= 8) {         // one division per group: the 8 elements lie in at most two kernel rows
+      int dy = (int)fastdiv((uint32_t)k0, g.dm, g.ds1, g.ds2);
+      int r = k0 - dy * g.kwC;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (r >= g.kwC) { r -= g.kwC; ++dy; }
+        const int off = off0 + r, ih = ih0 + dy;
+        float x = 0.0f;
+        if (k0 + j < g.K && ih >= 0 && ih < g.H && off >= 0 && off < g.WC) x = __ldg(img + (int64_t)ih * g.WC + off);
+        v[j] = x;
+        ++r;
+      }
     } else {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -157,12 +176,10 @@ __global__ void __launch_bounds__(256) im2col_quantize_kernel(const float* __res
       }
       *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(q) + row * ldq + k0) = make_uint4(o[0], o[1], o[2], o[3]);
     } else {
-      uint32_t lo = 0, hi = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        lo |= (uint32_t)(conv_code(v[j], inv_scale, qmax) & 0xff) << (8 * j);
-        hi |= (uint32_t)(conv_code(v[j + 4], inv_scale, qmax) & 0xff) << (8 * j);
-      }
+      const uint32_t lo = conv_pack4(conv_code(v[0], inv_scale, qmax), conv_code(v[1], inv_scale, qmax),
+                                     conv_code(v[2], inv_scale, qmax), conv_code(v[3], inv_scale, qmax));
+      const uint32_t hi = conv_pack4(conv_code(v[4], inv_scale, qmax), conv_code(v[5], inv_scale, qmax),
+                                     conv_code(v[6], inv_scale, qmax), conv_code(v[7], inv_scale, qmax));
       *reinterpret_cast<uint2*>(reinterpret_cast<int8_t*>(q) + row * ldq + k0) = make_uint2(lo, hi);
     }
   }
