@@ -117,6 +117,24 @@ def bert_layers(hidden: int, ffn: int, n_blocks: int) -> List[Layer]:
     return out
 
 
+def bert_layers_wide_qkv(hidden: int, ffn: int, n_blocks: int) -> List[Layer]:
+    """The same stand-in graph with the three projections of a block as ONE layer of
+    3*hidden output channels (rows 0..hidden-1 = Wq, then Wk, then Wv).  Wo reads the
+    V columns of that layer's output through src_col0 = 2*hidden; two tap layers read
+    the Q and K column slices, so every third of the wide output has a reader."""
+    out: List[Layer] = []
+    for blk in range(n_blocks):
+        base = 6 * blk
+        h_src = base - 1
+        out.append(Layer(f"b{blk}.qkv", 3 * hidden, hidden, src=h_src))
+        out.append(Layer(f"b{blk}.qtap", hidden, hidden, src=base, src_col0=0))
+        out.append(Layer(f"b{blk}.ktap", hidden, hidden, src=base, src_col0=hidden))
+        out.append(Layer(f"b{blk}.o", hidden, hidden, src=base, src_col0=2 * hidden))
+        out.append(Layer(f"b{blk}.ffn1", ffn, hidden, src=base + 3, act=ACT_GELU_TANH))
+        out.append(Layer(f"b{blk}.ffn2", hidden, ffn, src=base + 4))
+    return out
+
+
 def resnet50_layers(in_hw: int = 224, width: int = 64, n_classes: int = 1000,
                     blocks: Sequence[int] = (3, 4, 6, 3)) -> List[Layer]:
     """ResNet-50 v1.5 as NHWC im2col GEMMs (stride 2 sits in the 3x3 convolution).
@@ -227,6 +245,19 @@ def bert_stack(seed: int, m: int, hidden: int, ffn: int, n_blocks: int,
         bits = rng.choice(np.asarray(bit_choices, dtype=np.uint8), size=len(layers))
     accept = rng.random(n_accept) < 0.5 if n_accept else None
     return Workload(name, seed, layers, m, x, weights, bits=bits, accept=accept,
+                    meta={"hidden": hidden, "ffn": ffn, "n_blocks": n_blocks})
+
+
+def bert_stack_wide_qkv(seed: int, m: int, hidden: int, ffn: int, n_blocks: int,
+                        bit_choices: Sequence[int] = (4, 8, 16)) -> Workload:
+    """bert_stack's draws for the wide-projection graph (column-slice consumers)."""
+    rng = np.random.default_rng(seed)
+    layers = bert_layers_wide_qkv(hidden, ffn, n_blocks)
+    x = rng.standard_normal((m, hidden), dtype=np.float32)
+    weights = _normal_weights(rng, layers, lambda l: 0.02)
+    _apply_outliers(rng, weights)
+    bits = rng.choice(np.asarray(bit_choices, dtype=np.uint8), size=len(layers))
+    return Workload("bert_wide_qkv", seed, layers, m, x, weights, bits=bits,
                     meta={"hidden": hidden, "ffn": ffn, "n_blocks": n_blocks})
 
 

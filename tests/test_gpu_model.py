@@ -132,6 +132,40 @@ def test_bert_stack_teacher_forced(ctx, fuse, seed, m, hidden, ffn, blocks):
         ctx.set_fusion(True)
 
 
+@pytest.mark.parametrize("fuse", [True, False])
+def test_column_slice_consumers_teacher_forced(ctx, fuse):
+    """One wide projection layer (3h output channels) whose column thirds are read by three
+    consumers through src_col0 = 0, h, 2h: calibration maxima, input codes, accumulators and
+    outputs of every slice reader against the oracle, and the wide layer's thirds against three
+    separate projections with the same weight rows."""
+    ctx.set_fusion(fuse)
+    try:
+        h, ffn, m = 192, 768, 333
+        w = wl.bert_stack_wide_qkv(33, m, h, ffn, 2)
+        model, x = build(ctx, w)
+        act_g, w_amax = check_calibration(model, w)
+        for bits in (w.bits, [8] * len(w.layers), [4, 8, 16, 3, 16, 2] * 2, [16, 8, 4, 8, 8, 8] * 2):
+            ys = run_eval(ctx, model, w, x, bits)
+            teacher_forced_check(ctx, model, w, x, bits, ys, act_g, w_amax)
+        ys8 = run_eval(ctx, model, w, x, [8] * len(w.layers))
+        model.close()
+        # all-8: the wide layer's thirds equal three separate projections
+        sep = wl.Workload("sep", 33, wl.bert_layers(h, ffn, 2), m, w.x, [], bits=np.full(12, 8, np.uint8))
+        for blk in range(2):
+            wide = w.weights[6 * blk]
+            sep.weights += [wide[:h], wide[h:2 * h], wide[2 * h:]] + w.weights[6 * blk + 3:6 * blk + 6]
+        model_s, xs = build(ctx, sep)
+        ys_s = run_eval(ctx, model_s, sep, xs, sep.bits)
+        for blk in range(2):
+            for j in range(3):
+                assert torch.equal(ys8[6 * blk][:, j * h:(j + 1) * h], ys_s[6 * blk + j])
+            for j in (3, 4, 5):
+                assert torch.equal(ys8[6 * blk + j], ys_s[6 * blk + j])
+        model_s.close()
+    finally:
+        ctx.set_fusion(True)
+
+
 def test_fused_and_unfused_agree_bitwise_and_taps_are_optional(ctx):
     w = wl.bert_stack(21, 515, 128, 512, 2, bit_choices=(4, 8))
     model, x = build(ctx, w)

@@ -328,6 +328,146 @@ def test_resnet_chain_small_runs_and_residual_is_used():
     assert np.all(outs[c] >= 0)
 
 
+def test_e_qe_table_is_e_qe_elementwise():
+    sse = np.array([[4.0, 1.0, 0.25], [9.0, 0.0, 16.0], [1.0, 1.0, 1.0]])
+    sizes = [4, 9, 100]
+    amax = np.array([2.0, 0.5, 0.0], np.float32)           # the last tensor is all zero
+    tab = orc.e_qe_table(sse, sizes, amax)
+    # Eq. 2 by hand: sqrt(sse/n)/A
+    want = np.array([[0.5, 0.25, 0.125], [2.0, 0.0, 8.0 / 3.0], [0.0, 0.0, 0.0]])
+    np.testing.assert_allclose(tab, want, rtol=1e-15)
+    for t in range(3):
+        for j in range(3):
+            assert tab[t, j] == orc.e_qe(sse[t, j], sizes[t], float(amax[t]))
+
+
+@pytest.mark.parametrize("b", [3, 4, 8])
+def test_layer_forward_exact_on_grid_with_unequal_row_scales(b):
+    """Inputs and weights that already lie on their b-bit grids with power-of-two scales: every
+    step of the quantized layer is then exact, so its output must equal the real product bit for
+    bit.  The weight rows have maxima 2^8 apart, so a per-row scale taken from the wrong row, a
+    per-tensor weight scale, a transposed operand or a dropped activation scale all fail."""
+    rng = np.random.default_rng(40 + b)
+    qm = orc.qmax(b)
+    M, K, N = 9, 24, 5
+    cx = rng.integers(-qm, qm + 1, (M, K)).astype(np.float64)
+    cx[2, 7] = -qm                                         # the activation maximum
+    cw = rng.integers(-qm, qm + 1, (N, K)).astype(np.float64)
+    cw[np.arange(N), (3 * np.arange(N) + 1) % K] = qm * np.array([1, -1, 1, -1, 1])   # every row reaches +-qmax
+    e_x = -4
+    e_w = np.array([-3, 1, -7, 0, -5])
+    x = (cx * 2.0 ** e_x).astype(np.float32)
+    w = (cw * 2.0 ** e_w[:, None]).astype(np.float32)
+    lay = wl.Layer("l", N, K)
+    taps = {}
+    y = orc.layer_forward(lay, w, x, b, orc.absmax(x), orc.absmax(w, orc.PER_ROW), taps=taps)
+    np.testing.assert_array_equal(taps["qx"], cx.astype(np.int8))
+    np.testing.assert_array_equal(taps["qw"], cw.astype(np.int8))
+    np.testing.assert_array_equal(taps["scale_w"], (2.0 ** e_w).astype(np.float32))
+    assert taps["scale_x"] == np.float32(2.0 ** e_x)
+    want = x.astype(np.float64) @ w.astype(np.float64).T   # exact: integers times powers of two
+    np.testing.assert_array_equal(y.astype(np.float64), want)
+
+
+def test_layer_forward_shortcut_relu_and_clip_by_hand():
+    """2 x 2 x 2 case written out: the shortcut is added before the ReLU, and an input beyond the
+    CALIBRATED maximum is clipped (the activation scale is the calibrated one, not the input's)."""
+    lay = wl.Layer("l", 2, 2, act=orc.ACT_RELU)
+    b = 4                                                  # qmax 7
+    x = np.array([[1.0, -0.5], [3.5, 0.25]], np.float32)   # calibrated max 1.75 -> scale 0.25; 3.5 clips to 7
+    w = np.array([[7.0, -7.0], [0.5, 3.5]], np.float32)    # row maxima 7 and 3.5 -> scales 1 and 0.5
+    res = np.array([[-30.0, 0.125], [1.0, -100.0]], np.float32)
+    # codes: x -> [[4, -2], [7, 1]];  w -> [[7, -7], [1, 7]]
+    # acc  = [[4*7 + 2*7, 4*1 - 2*7], [7*7 - 1*7, 7*1 + 1*7]] = [[42, -10], [42, 14]]
+    # y    = acc * 0.25 * [1, 0.5]   = [[10.5, -1.25], [10.5, 1.75]]
+    # + res                          = [[-19.5, -1.125], [11.5, -98.25]];  ReLU -> [[0, 0], [11.5, 0]]
+    taps = {}
+    y = orc.layer_forward(lay, w, x, b, np.float32(1.75), orc.absmax(w, orc.PER_ROW), residual=res, taps=taps)
+    np.testing.assert_array_equal(taps["qx"], np.array([[4, -2], [7, 1]], np.int8))
+    np.testing.assert_array_equal(taps["acc"], np.array([[42, -10], [42, 14]], np.int32))
+    np.testing.assert_array_equal(y, np.array([[0.0, 0.0], [11.5, 0.0]], np.float32))
+    lay_none = wl.Layer("l", 2, 2)
+    y2 = orc.layer_forward(lay_none, w, x, b, np.float32(1.75), orc.absmax(w, orc.PER_ROW), residual=res)
+    np.testing.assert_array_equal(y2, np.array([[-19.5, -1.125], [11.5, -98.25]], np.float32))
+
+
+def test_conv_pool_reshape_chain_matches_library():
+    """layer_input's convolution / pooling / reshape branch, value by value: a 7x7/2 stem, a 3x3/2
+    max-pool, a 1x1 convolution, a 3x3/2 convolution and a global-average-pooled linear layer on a
+    NON-square image, every layer at 16 bit.  Inputs and weights are small integers, so every
+    product, sum and bf16 rounding is exact and the library's convolutions must agree bit for bit.
+    A swapped height/width in the reshape, a wrong pooling window or a wrong patch order fails."""
+    F = torch.nn.functional
+    rng = np.random.default_rng(77)
+    B, H, W = 2, 20, 14
+    L = [
+        wl.Layer("stem", 6, 7 * 7 * 3, src=-1, act=wl.ACT_RELU, kh=7, kw=7, stride=2, pad=3, in_h=H, in_w=W, in_c=3,
+                 src_h=H, src_w=W),                                                        # -> 10 x 7
+        wl.Layer("p1", 4, 6, src=0, act=wl.ACT_RELU, kh=1, kw=1, stride=1, pad=0, in_h=5, in_w=4, in_c=6,
+                 pool_before=wl.POOL_MAX3S2, src_h=10, src_w=7),                            # pool -> 5 x 4
+        wl.Layer("c3", 5, 3 * 3 * 4, src=1, act=wl.ACT_NONE, kh=3, kw=3, stride=2, pad=1, in_h=5, in_w=4, in_c=4,
+                 src_h=5, src_w=4),                                                        # -> 3 x 2
+        wl.Layer("fc", 3, 5, src=2, pool_before=wl.POOL_GLOBAL_AVG, src_h=3, src_w=2),
+    ]
+    x = rng.integers(-3, 4, (B, H, W, 3)).astype(np.float32)
+    ws = [rng.integers(-2, 3, (l.n_out, l.k_in)).astype(np.float32) for l in L]
+    outs = orc.eval_config(L, ws, [16] * 4, x, [None] * 4, [None] * 4)
+
+    def bf(t):
+        return t.float().to(torch.bfloat16).double()
+
+    def conv(t, w, lay):
+        w4 = torch.from_numpy(w).double().reshape(lay.n_out, lay.kh, lay.kw, lay.in_c).permute(0, 3, 1, 2)
+        return F.conv2d(bf(t), bf(w4), stride=lay.stride, padding=lay.pad).float()
+
+    t = torch.from_numpy(x).permute(0, 3, 1, 2)                       # NCHW
+    y0 = torch.relu(conv(t, ws[0], L[0]))
+    assert y0.shape[2:] == (10, 7)
+    y1 = torch.relu(conv(F.max_pool2d(y0, 3, 2, 1), ws[1], L[1]))
+    assert y1.shape[2:] == (5, 4)
+    y2 = conv(y1, ws[2], L[2])
+    assert y2.shape[2:] == (3, 2)
+    y3 = (bf(y2.double().mean(dim=(2, 3)).float()) @ bf(torch.from_numpy(ws[3])).T).float()
+    for got, want in zip(outs[:3], (y0, y1, y2)):
+        np.testing.assert_array_equal(got, want.permute(0, 2, 3, 1).reshape(-1, want.shape[1]).numpy())
+    np.testing.assert_array_equal(outs[3], y3.numpy())
+    assert float(np.abs(outs[2]).max()) > 100                        # the chain is not trivially zero
+
+
+def test_column_slice_consumers_equal_separate_projections():
+    """src_col0: a layer of 3h output channels whose thirds are read by three consumers must give
+    what three separate h-channel layers with the same weight rows give (rows of a product are
+    independent, per-row weight scales do not mix rows).  Ignoring src_col0, or slicing rows
+    instead of columns, makes the consumer of the last third read the wrong tensor."""
+    h, ffn, m = 16, 48, 21
+    ww = wl.bert_stack_wide_qkv(31, m, h, ffn, 2, bit_choices=(4, 8))
+    sep = wl.bert_layers(h, ffn, 2)
+    w_sep, bits_sep = [], []
+    for blk in range(2):
+        wide = ww.weights[6 * blk]
+        w_sep += [wide[:h], wide[h:2 * h], wide[2 * h:], ww.weights[6 * blk + 3], ww.weights[6 * blk + 4], ww.weights[6 * blk + 5]]
+        bq = int(ww.bits[6 * blk])
+        bits_sep += [bq, bq, bq] + [int(v) for v in ww.bits[6 * blk + 3:6 * blk + 6]]
+    act_w, wam_w = orc.calibrate_model(ww.layers, ww.weights, ww.x)
+    act_s, wam_s = orc.calibrate_model(sep, w_sep, ww.x)
+    outs_w = orc.eval_config(ww.layers, ww.weights, ww.bits, ww.x, act_w, wam_w)
+    outs_s = orc.eval_config(sep, w_sep, bits_sep, ww.x, act_s, wam_s)
+    for blk in range(2):
+        base = 6 * blk
+        wide = outs_w[base]
+        for j in range(3):
+            np.testing.assert_array_equal(wide[:, j * h:(j + 1) * h], outs_s[base + j])
+        for j in (3, 4, 5):
+            np.testing.assert_array_equal(outs_w[base + j], outs_s[base + j])
+            assert act_w[base + j] == act_s[base + j]
+        # what each slice reader was fed, by manual slicing
+        for j, lay_idx in enumerate((base + 1, base + 2, base + 3)):
+            xin = orc.layer_input(ww.layers, lay_idx, ww.x, outs_w)
+            np.testing.assert_array_equal(xin, wide[:, j * h:(j + 1) * h])
+            assert act_w[lay_idx] == np.max(np.abs(orc.eval_config(ww.layers, ww.weights, [16] * 12, ww.x, act_w, wam_w)[base][:, j * h:(j + 1) * h]))
+    assert not np.array_equal(outs_w[0][:, :h], outs_w[0][:, 2 * h:])
+
+
 # ----------------------------------------------------------------------- tables and sequences
 
 def test_layer_tables_match_table1_sizes():
