@@ -43,7 +43,6 @@ enum {
   QCFG_EARCH = 7,      /* device is not sm_100                                      */
   QCFG_ECUDA = 8,      /* a CUDA runtime/driver call failed; see qcfg_last_error    */
   QCFG_ETIMEOUT = 9,   /* a bounded device-side wait gave up                        */
-  QCFG_EUNIMPL = 10,   /* feature not available in this build                       */
   QCFG_ESTATE = 11     /* call order (e.g. evaluation before calibration)           */
 };
 enum { QCFG_PER_TENSOR = 0, QCFG_PER_ROW = 1 };
@@ -52,7 +51,7 @@ enum { QCFG_POOL_NONE = 0, QCFG_POOL_MAX3S2 = 1, QCFG_POOL_GLOBAL_AVG = 2 };
 
 /* One "tensor" of the bit configuration: a linear or convolution layer whose weight and
  * input activation share one bit width (Algorithms 1 and 2 index the configuration by
- * layer; Table 1: "same bit-precision for all their weights and activations").           */
+ * layer; Table 1's uniform rows likewise use one width for a layer's weight and input).  */
 typedef struct qcfg_layer {
   const float* w_dev;    /* [n_out][k_in] fp32, borrowed for the model's lifetime          */
   int64_t n_out, k_in;
@@ -77,6 +76,12 @@ int qcfg_destroy(qcfg_ctx* ctx);
 /* Synchronises `stream`, then returns and clears the device error word:
  * QCFG_OK, QCFG_ETIMEOUT, QCFG_ENONFINITE or QCFG_ECUDA.                                  */
 int qcfg_sync_status(qcfg_ctx* ctx, void* stream);
+/* Self-test of the failure path of the kernels' bounded waits (every device-side wait on a
+ * barrier gives up after a time limit instead of hanging): enqueues a one-thread kernel that
+ * waits on a barrier nothing arrives on, with a limit of limit_ns nanoseconds (1 .. 1e8).  The
+ * wait runs out, the kernel sets the time-out bit of the context's error word and ends normally;
+ * the next qcfg_sync_status returns QCFG_ETIMEOUT and clears it.  Nothing else is touched.   */
+int qcfg_selftest_wait_timeout(qcfg_ctx* ctx, uint64_t limit_ns, void* stream);
 /* Library-owned, NUL-terminated description of the last non-OK status of this context.   */
 const char* qcfg_last_error(qcfg_ctx* ctx);
 /* Number of kernels this context has launched since creation (for accounting).            */
@@ -84,7 +89,8 @@ int64_t qcfg_launch_count(qcfg_ctx* ctx);
 
 /* Switches the fusion of the consumer's quantize step into the producing GEMM's epilogue
  * (default on).  Off: every layer's fp32 output is written and re-read by a separate quantize
- * kernel; results are bit-identical either way.                                           */
+ * kernel; results are bit-identical either way for finite values (a NaN, which calibration
+ * rejects, is clamped to a code of either sign depending on the path).                     */
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled);
 /* Switches the two-CTA GEMM tiles (256 rows per CTA pair, cta_group::2; default on, used for
  * outputs wider than 128 columns and more than 128 rows).  Off: every tile is 128 rows on one

@@ -18,11 +18,12 @@ OK = 0
 PER_TENSOR, PER_ROW = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
 SEARCH_BISECTION, SEARCH_GREEDY = 0, 1
-STATUS_NAMES = ["OK", "EINVAL", "EBITS", "ESHAPE", "EALIGN", "ENOMEM", "ENONFINITE", "EARCH", "ECUDA",
-                "ETIMEOUT", "EUNIMPL", "ESTATE"]
-EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT, EUNIMPL, ESTATE = range(1, 12)
+STATUS_NAMES = {0: "OK", 1: "EINVAL", 2: "EBITS", 3: "ESHAPE", 4: "EALIGN", 5: "ENOMEM", 6: "ENONFINITE", 7: "EARCH",
+                8: "ECUDA", 9: "ETIMEOUT", 11: "ESTATE"}
+EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT = range(1, 10)
+ESTATE = 11
 
-EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error", "qcfg_launch_count",
+EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_selftest_wait_timeout", "qcfg_last_error", "qcfg_launch_count",
            "qcfg_set_fusion", "qcfg_set_pair_tiles", "qcfg_set_grouping", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
@@ -31,7 +32,7 @@ EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_last_error",
 
 class QcfgError(RuntimeError):
     def __init__(self, status: int, msg: str = ""):
-        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        name = STATUS_NAMES.get(status, str(status))
         super().__init__(f"QCFG_{name}: {msg}")
         self.status = status
 
@@ -60,6 +61,7 @@ def load_library() -> C.CDLL:
         "qcfg_create": [C.POINTER(vp), ci],
         "qcfg_destroy": [vp],
         "qcfg_sync_status": [vp, vp],
+        "qcfg_selftest_wait_timeout": [vp, C.c_uint64, vp],
         "qcfg_set_fusion": [vp, ci],
         "qcfg_set_pair_tiles": [vp, ci],
         "qcfg_set_grouping": [vp, ci],
@@ -144,6 +146,9 @@ class Context:
 
     def sync_status(self, stream=None) -> int:
         return int(self.lib.qcfg_sync_status(self.h, _stream(stream)))
+
+    def selftest_wait_timeout(self, limit_ns: int, stream=None):
+        self._check(self.lib.qcfg_selftest_wait_timeout(self.h, int(limit_ns), _stream(stream)))
 
     def check_sync(self, stream=None):
         self._check(self.sync_status(stream))

@@ -436,6 +436,7 @@ int qcfg_create(qcfg_ctx** out, int device) {
     return QCFG_ENOMEM;
   }
   int rc = gemm_init(&h->c);
+  if (!rc) rc = sweep_init(&h->c);
   if (rc) { cudaFree(h->c.err_dev); delete h; return rc; }
   *out = h;
   return QCFG_OK;
@@ -465,6 +466,12 @@ int qcfg_sync_status(qcfg_ctx* ctx, void* stream) {
     if (w & ERR_NONFINITE) return set_error(c, QCFG_ENONFINITE, "non-finite value found on the device");
   }
   return QCFG_OK;
+}
+
+int qcfg_selftest_wait_timeout(qcfg_ctx* ctx, uint64_t limit_ns, void* stream) {
+  if (!ctx) return QCFG_EINVAL;
+  if (limit_ns == 0 || limit_ns > 100000000ull) return set_error(&ctx->c, QCFG_EINVAL, "selftest: limit must be 1 ns .. 100 ms");
+  return launch_wait_timeout(&ctx->c, limit_ns, (cudaStream_t)stream);
 }
 
 const char* qcfg_last_error(qcfg_ctx* ctx) { return ctx ? ctx->c.msg : "null context"; }
@@ -886,34 +893,51 @@ int qcfg_search(qcfg_ctx* ctx, qcfg_model* model, int algorithm, const int32_t* 
   if (rc) return rc;
   S.ys[n - 1] = (float*)M->search_out.p;
 
-  std::vector<int> ll(order, order + n);
+  // `config` is the working configuration; `candidates` are the layers still eligible for a lower
+  // width, least sensitive first.  Both searches lower widths one value of `lower` at a time.
+  std::vector<uint8_t>& config = w;
+  std::vector<int> candidates(order, order + n);
+  // the working configuration with the first `count` candidates set to `width`
+  auto with_prefix = [&](int count, int width) {
+    std::vector<uint8_t> trial(config);
+    for (int i = 0; i < count; ++i) trial[candidates[i]] = (uint8_t)width;
+    return trial;
+  };
   if (algorithm == QCFG_SEARCH_BISECTION) {
-    for (int b : lower) {
-      int thr = (int)ll.size() / 2, upl = (int)ll.size(), lowl = 0;
-      for (;;) {
-        std::vector<uint8_t> lw(w);
-        for (int i = 0; i < thr; ++i) lw[ll[i]] = (uint8_t)b;
-        const double a = search_evaluate(S, lw);
+    // Algorithm 1: binary search for the longest prefix of the candidates that can take `width`.
+    // `passing` is the longest prefix known to meet the target, `failing` the shortest known not
+    // to (or one past the list); the probe moves halfway (floor) towards whichever bound is open
+    // and the search ends when it stops moving.  The prefix written is `passing`.
+    for (int width : lower) {
+      const int count = (int)candidates.size();
+      int passing = 0, failing = count, probe = count / 2;
+      bool moved = true;
+      while (moved) {
+        const double fidelity = search_evaluate(S, with_prefix(probe, width));
         if (S.rc) return S.rc;
-        const int old = thr;
-        if (a >= target) { lowl = thr; thr = thr + (upl - thr) / 2; }
-        else { upl = thr; thr = thr - (thr - lowl) / 2; }
-        if (thr == old) break;
+        int next;
+        if (fidelity >= target) { passing = probe; next = probe + (failing - probe) / 2; }
+        else { failing = probe; next = probe - (probe - passing) / 2; }
+        moved = next != probe;
+        probe = next;
       }
-      for (int i = 0; i < lowl; ++i) w[ll[i]] = (uint8_t)b;
-      ll.resize(lowl);
+      config = with_prefix(passing, width);
+      candidates.resize(passing);
     }
   } else {
-    for (int b : lower) {
-      std::vector<int> ql;
-      for (int l : ll) {
-        const uint8_t last = w[l];
-        w[l] = (uint8_t)b;
-        const double a = search_evaluate(S, w);
+    // Algorithm 2: try `width` on one candidate at a time, keeping each change that meets the
+    // target; only the layers that took this width stay candidates for the next one.
+    for (int width : lower) {
+      std::vector<int> kept;
+      for (int layer : candidates) {
+        const uint8_t before = config[layer];
+        config[layer] = (uint8_t)width;
+        const double fidelity = search_evaluate(S, config);
         if (S.rc) return S.rc;
-        if (a >= target) ql.push_back(l); else w[l] = last;
+        if (fidelity >= target) kept.push_back(layer);
+        else config[layer] = before;
       }
-      ll.swap(ql);
+      candidates.swap(kept);
     }
   }
   memcpy(bits_out, w.data(), n);

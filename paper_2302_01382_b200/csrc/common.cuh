@@ -53,6 +53,7 @@ int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, 
                            int pad, float inv_scale, int bits, void* q, int64_t ldq, cudaStream_t st);
 
 // ----- sweep.cu -----------------------------------------------------------------------
+int sweep_init(Ctx* ctx);   // per-device kernel attributes
 int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
                  int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse,
                  float* absmax, cudaStream_t st);
@@ -88,6 +89,7 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st);
 bool gemm_groupable(const GemmArgs& a, const GemmArgs& b);
 int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st);
 int gemm_init(Ctx* ctx);   // resolves the tensor-map encoder, sets smem attributes
+int launch_wait_timeout(Ctx* ctx, uint64_t limit_ns, cudaStream_t st);
 
 // ----- small device helpers -----------------------------------------------------------
 __device__ __forceinline__ unsigned warp_max_u(unsigned v) {

@@ -101,7 +101,8 @@ __device__ __forceinline__ uint64_t global_timer() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA should give up (this or another wait timed out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* err) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* err,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   uint64_t t0 = 0;
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -109,7 +110,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       uint64_t now = global_timer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         atomicOr(err, ERR_TIMEOUT);
         *abort_flag = 1;
         return false;
@@ -790,7 +791,27 @@ bool make_out_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
   return r == CUDA_SUCCESS;
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on, with
+// a caller-chosen limit; the wait gives up, sets the time-out bit of the error word and the
+// kernel ends normally.
+__global__ void wait_timeout_kernel(uint64_t limit_ns, unsigned* err) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    (void)mbar_wait(smem_u32(&bar), 0, &abort_flag, err, limit_ns);
+  }
+}
+
 }  // namespace
+
+int launch_wait_timeout(Ctx* ctx, uint64_t limit_ns, cudaStream_t st) {
+  wait_timeout_kernel<<<1, 32, 0, st>>>(limit_ns, err_word(ctx));
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "wait self-test launch");
+}
 
 int gemm_init(Ctx* ctx) {
   if (!g_encode) {

@@ -299,15 +299,30 @@ template <int V>
 void launch_rows(const SweepDesc* d, int n, int items, int per_tensor, const float* amax, int jlo, int jhi,
                  double* partial, cudaStream_t st) {
   constexpr size_t smem = (size_t)kRing * V * kThreads * sizeof(float4);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(sweep_rows_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    attr_set = true;
-  }
   sweep_rows_kernel<V><<<items, kThreads, smem, st>>>(d, n, per_tensor, amax, jlo, jhi, partial);
 }
 
+template <int V>
+cudaError_t set_rows_smem() {
+  return cudaFuncSetAttribute(sweep_rows_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)((size_t)kRing * V * kThreads * sizeof(float4)));
+}
+
 }  // namespace
+
+// The shared-memory opt-in of a kernel is a per-device attribute: set for every variant whenever a
+// context is created (the context's device is current then).
+int sweep_init(Ctx* ctx) {
+  cudaError_t e = set_rows_smem<1>();
+  if (e == cudaSuccess) e = set_rows_smem<2>();
+  if (e == cudaSuccess) e = set_rows_smem<3>();
+  if (e == cudaSuccess) e = set_rows_smem<4>();
+  if (e == cudaSuccess) e = set_rows_smem<5>();
+  if (e == cudaSuccess) e = set_rows_smem<6>();
+  if (e == cudaSuccess) e = set_rows_smem<7>();
+  if (e == cudaSuccess) e = set_rows_smem<8>();
+  return check_cuda(ctx, e, "sweep smem attribute");
+}
 
 int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols, int32_t n_tensors,
                  int granularity, int b_lo, int b_hi, double* sse, float* absmax, cudaStream_t st) {

@@ -294,3 +294,41 @@ def test_argument_errors_leave_outputs_untouched(ctx):
     assert e.value.status == q.EALIGN
     assert "16-byte" in ctx.last_error()
     assert ctx.sync_status() == q.OK
+
+
+# ----------------------------------------------------------------------------- device-side faults
+
+def test_bounded_wait_gives_up_and_the_context_stays_usable(ctx):
+    """A device wait whose barrier is never signalled runs into its limit (1 ms here), reports
+    QCFG_ETIMEOUT through the error word, and leaves the context able to run a correct GEMM."""
+    import paper_2302_01382_b200 as q
+    assert ctx.sync_status() == q.OK
+    ctx.selftest_wait_timeout(1_000_000)
+    assert ctx.sync_status() == q.ETIMEOUT
+    assert "wait" in ctx.last_error()
+    assert ctx.sync_status() == q.OK                  # the error word was cleared by the read
+    rng = np.random.default_rng(5)
+    qx = rng.integers(-127, 128, (200, 64), dtype=np.int8)
+    qw = rng.integers(-127, 128, (48, 64), dtype=np.int8)
+    _, acc = ctx.gemm_i8(dev(qx), dev(qw), 64, 1.0, None, want_y=False, want_acc=True)
+    assert ctx.sync_status() == q.OK
+    np.testing.assert_array_equal(host(acc), orc.int_gemm(qx, qw))
+    with pytest.raises(q.QcfgError) as e:
+        ctx.selftest_wait_timeout(0)
+    assert e.value.status == q.EINVAL
+
+
+def test_second_context_sweeps_wide_rows():
+    """The sweep's shared-memory opt-in is set per context: a context created after another one
+    has already swept still runs the variants that need more than 48 KB of shared memory."""
+    import paper_2302_01382_b200 as q
+    rng = np.random.default_rng(6)
+    x = rng.standard_normal((40, 768)).astype(np.float32)
+    so, ao = orc.quant_error_sweep([x])
+    for _ in range(2):
+        c = q.Context(0)
+        sse, amax = c.quant_error_sweep([dev(x)])
+        c.check_sync()
+        np.testing.assert_allclose(host(sse), so, rtol=1e-5)
+        np.testing.assert_array_equal(host(amax), ao)
+        c.close()
