@@ -37,7 +37,8 @@ TOKENS = 32 * 384
 WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
 # DRAM bytes (read + write) per int8 GEMM launch from the ncu capture summarised in
 # profiles/gemm_int8_bert_base_block.md; set to None whenever the GEMM kernel changes.
-GEMM_TRAFFIC_BYTES = 27.6e6
+GEMM_TRAFFIC_BYTES = None
+DATASHEET_INT8_TOPS = 4500.0      # B200 dense int8, vendor datasheet (an outside figure)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -236,6 +237,82 @@ class Job:
             main.wait_stream(self.copy_stream)
 
 
+def timed_evals(torch, ctx, model, configs, x, m, ys, reps: int):
+    """Device time of `reps` passes over `configs` (inputs resident), plus the GEMM kernels' own
+    time stamps (first CTA start to last CTA end of every launch) from the same passes."""
+    for bits in configs[:2]:
+        model.eval_config(bits, x, m, ys)
+    ctx.check_sync()
+    l0 = ctx.launch_count()
+    ctx.profile_enable(2)
+    ctx.profile_read(0); ctx.profile_read(1)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        for bits in configs:
+            model.eval_config(bits, x, m, ys)
+    e1.record()
+    torch.cuda.synchronize()
+    i_ms, i_n, i_ops = ctx.profile_read(0)
+    b_ms, b_n, b_ops = ctx.profile_read(1)
+    ctx.profile_enable(0)
+    n = reps * len(configs)
+    ms = e0.elapsed_time(e1) / n
+    k_ms = i_ms + b_ms
+    return {"evals_per_s": 1e3 / ms, "ms_per_eval": ms, "evals_timed": n,
+            "gemm_tops": (i_ops + b_ops) / (k_ms * 1e-3) / 1e12 if k_ms else None,
+            "gemm_int8_tops": i_ops / (i_ms * 1e-3) / 1e12 if i_ms else None,
+            "gemm_bf16_tflops": b_ops / (b_ms * 1e-3) / 1e12 if b_ms else None,
+            "gemm_ms_per_eval": k_ms / n, "launches_per_eval": (ctx.launch_count() - l0) / n}
+
+
+def other_workloads(torch, q, ctx, peaks):
+    """Short timed legs of the other four workloads (inputs resident, CUDA events)."""
+    out = {}
+
+    def leg(name, w, configs, reps, sweep=False):
+        weights = [torch.from_numpy(a).cuda() for a in w.weights]
+        x = torch.from_numpy(w.x).cuda()
+        model = q.Model(ctx, w.layers, weights)
+        model.calibrate_model(x, w.m)
+        rank = None
+        res = {}
+        if sweep:
+            sse, amax = ctx.quant_error_sweep(weights)
+            sizes = np.array([a.size for a in w.weights], np.float64)
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record()
+            for _ in range(5):
+                ctx.quant_error_sweep(weights, sse=sse, absmax=amax)
+            s1.record()
+            torch.cuda.synchronize()
+            nbytes = 4.0 * float(sizes.sum())
+            res["sweep_gbs"] = nbytes / (s0.elapsed_time(s1) / 5 * 1e-3) / 1e9
+            res["sweep_frac_hbm"] = res["sweep_gbs"] / peaks["hbm_gbs"]
+            eqe = np.sqrt(sse.cpu().numpy()[:, 2] / sizes) / np.maximum(amax.cpu().numpy().astype(np.float64), 1e-30)
+            rank = np.argsort(eqe, kind="stable")
+        cfgs = configs(rank) if callable(configs) else configs
+        rows_out = wl.layer_rows(w.layers, len(w.layers) - 1, w.m)
+        ys = [None] * (len(w.layers) - 1) + [torch.empty((rows_out, w.layers[-1].n_out), device="cuda")]
+        res.update(timed_evals(torch, ctx, model, cfgs, x, w.m, ys, reps))
+        res["bits"] = sorted(set(int(b) for c in cfgs for b in c))
+        res["layers"] = len(w.layers)
+        out[name] = res
+        model.close()
+        del weights, x, ys
+        torch.cuda.empty_cache()
+
+    w1 = wl.tiny_mlp()
+    leg("tiny_mlp_64x256", w1, [w1.bits], 200, sweep=True)
+    w2 = wl.bert_base_block()
+    leg("bert_base_block_3072_tokens_mixed_4_8_16", w2, [w2.bits], 50, sweep=True)
+    w4 = wl.resnet50()
+    leg("resnet50_batch128_bits_4_6_8_first_last_16", w4, [w4.bits], 5)
+    w5 = wl.bert_large_x24()
+    leg("bert_large_x24_6144_tokens_bisection8", w5, lambda rank: wl.bisection_sequence(rank, w5.accept, 108, 8), 2, sweep=True)
+    return out
+
+
 def run_gpu(args):
     import torch
     import paper_2302_01382_b200 as q
@@ -259,11 +336,14 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---------------- device-resident timing (value): no instrumentation inside the region
+    # ---------------- device-resident timing (value).  The GEMM kernels stamp their own start and
+    # end times (two atomics per CTA) in this same pass; nothing else is instrumented.
     for _ in range(args.warmup):
         job.step()
     ctx.check_sync()
     launches0 = ctx.launch_count()
+    ctx.profile_enable(2)
+    ctx.profile_read(0); ctx.profile_read(1)
     sampler = ClockSampler(dev_index)
     sampler.start()
     barrier()
@@ -278,25 +358,27 @@ def run_gpu(args):
     clocks = sampler.stop()
     launches = ctx.launch_count() - launches0
     value = world * N_EVALS * args.steps / (ms_total * 1e-3)
+    g_ms, g_n, g_ops = ctx.profile_read(0)
+    b_ms, b_n, b_ops = ctx.profile_read(1)
+    ctx.profile_enable(0)
 
-    # ---------------- the same steps again with CUDA events around every GEMM launch (roofline of
-    # the dominant kernel; the events serialise launches that otherwise overlap, so this pass is
-    # not the one `value` comes from)
-    ctx.profile_enable(True)
+    # ---------------- one more step with CUDA events around every launch: shares of the kernel
+    # classes (the events serialise launches that otherwise overlap, so this step is slower)
+    ctx.profile_enable(1)
     ctx.profile_read(0); ctx.profile_read(1); ctx.profile_read(2)
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record()
-    for _ in range(args.steps):
-        job.step()
+    job.step()
     p1.record()
     torch.cuda.synchronize()
-    g_ms, g_n, g_ops = ctx.profile_read(0)
-    b_ms, b_n, b_ops = ctx.profile_read(1)
-    o_ms, o_n, _ = ctx.profile_read(2)
-    ctx.profile_enable(False)
+    eg_ms, eg_n, eg_ops = ctx.profile_read(0)
+    eb_ms, _, _ = ctx.profile_read(1)
+    eo_ms, eo_n, _ = ctx.profile_read(2)
+    ctx.profile_enable(0)
     instrumented_ms = p0.elapsed_time(p1)
 
-    # ---------------- sweep alone (sub-metric), L2 flushed by its own 340 MB input
+    # ---------------- sweep alone (sub-metric), L2 flushed by its own 340 MB input: a burst of 10
+    # calls, then a loop of about half a second with the SM clock sampled
     sw0, sw1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n_sw = 10
     sw0.record()
@@ -305,8 +387,46 @@ def run_gpu(args):
     sw1.record()
     torch.cuda.synchronize()
     sweep_ms = sw0.elapsed_time(sw1) / n_sw
-    sweep_bytes = 4.0 * float(job.sizes.sum())
+    sweep_elems = float(job.sizes.sum())
+    sweep_bytes = 4.0 * sweep_elems
     sweep_gbs = sweep_bytes / (sweep_ms * 1e-3) / 1e9
+    n_long = max(200, int(500.0 / sweep_ms))
+    s_sampler = ClockSampler(dev_index)
+    s_sampler.start()
+    sw0.record()
+    for _ in range(n_long):
+        ctx.quant_error_sweep(job.weights, q.PER_ROW, 2, 8, sse=job.sse, absmax=job.amax)
+    sw1.record()
+    torch.cuda.synchronize()
+    s_clocks = s_sampler.stop()
+    sweep_long_ms = sw0.elapsed_time(sw1) / n_long
+    sweep_long_gbs = sweep_bytes / (sweep_long_ms * 1e-3) / 1e9
+    sweep_clock = s_clocks.get("sm_mhz") or clocks.get("sm_mhz") or peaks.get("sm_max_mhz", 1965.0)
+    alu_peak = 148 * 128 * sweep_clock * 1e6          # fp32 lane-operations per second at the sampled clock
+    alu_frac = 28.0 * sweep_elems / (sweep_long_ms * 1e-3) / alu_peak
+    hbm_frac_long = sweep_long_gbs / peaks["hbm_gbs"]
+
+    # ---------------- the build's own ceiling for the int8 GEMM: a large square problem with int8
+    # output, timed by the kernel's stamps in this process
+    own = None
+    if world == 1:
+        mq, nq, kq = 12288, 4096, 4096
+        gq = torch.Generator(device="cuda").manual_seed(0)
+        qa = torch.randint(-127, 128, (mq, kq), dtype=torch.int8, device="cuda", generator=gq)
+        qb = torch.randint(-127, 128, (nq, kq), dtype=torch.int8, device="cuda", generator=gq)
+        swq = torch.full((nq,), 1e-4, device="cuda")
+        oq = torch.empty((mq, nq), dtype=torch.int8, device="cuda")
+        for _ in range(3):
+            ctx.gemm_i8_requant(qa, qb, kq, 0.01, swq, q.ACT_NONE, 3.0, 8, out=oq)
+        ctx.check_sync()
+        ctx.profile_enable(2); ctx.profile_read(0)
+        for _ in range(20):
+            ctx.gemm_i8_requant(qa, qb, kq, 0.01, swq, q.ACT_NONE, 3.0, 8, out=oq)
+        torch.cuda.synchronize()
+        o_ms, o_n, o_ops = ctx.profile_read(0)
+        ctx.profile_enable(0)
+        own = {"m": mq, "n": nq, "k": kq, "tops": o_ops / (o_ms * 1e-3) / 1e12, "launches": int(o_n)}
+        del qa, qb, oq
 
     # ---------------- end to end: host buffers, copies inside the timed region
     e2e = None
@@ -314,7 +434,7 @@ def run_gpu(args):
         host_x = torch.from_numpy(w.x).pin_memory()
         host_out = [torch.empty((w.m, w.layers[-1].n_out), dtype=torch.float32).pin_memory() for _ in range(2)]
         x_dev = torch.empty_like(job.x)
-        e2e_steps = max(1, min(args.steps, 3))
+        e2e_steps = max(1, args.steps)
         barrier()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
@@ -343,9 +463,22 @@ def run_gpu(args):
         search = {"algorithm": "greedy", "bs": [8, 4], "target_fidelity": 0.9, "evals": int(n_s), "ms": 1e3 * dt,
                   "evals_per_s": n_s / dt, "layers_at_4_bit": int(sum(1 for b in bits_s if b == 4))}
 
+    # ---------------- the other four workloads
+    workloads = None
+    if world == 1 and not args.no_workloads:
+        job.model.close()
+        del job
+        torch.cuda.empty_cache()
+        workloads = other_workloads(torch, q, ctx, peaks)
+
     if rank == 0:
-        int8_peak = 2.0 * peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])
-        achieved = (g_ops / max(g_n, 1)) / (g_ms / max(g_n, 1) * 1e-3) / 1e12 if g_n else 0.0
+        sustained2 = 2.0 * peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])
+        burst2 = 2.0 * peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])
+        achieved = g_ops / (g_ms * 1e-3) / 1e12 if g_ms else 0.0
+        frac_of = {"2x_bf16_cublas_sustained": achieved / sustained2, "2x_bf16_cublas_burst": achieved / burst2,
+                   "datasheet_dense_int8_4500": achieved / DATASHEET_INT8_TOPS}
+        if own:
+            frac_of["own_large_square_int8"] = achieved / own["tops"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -355,17 +488,32 @@ def run_gpu(args):
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": e2e, "launches_before_timed": int(launches0),
-            "roofline": {"kernel": "gemm_kernel<int8>", "bound": "tensor", "achieved": achieved, "peak": int8_peak,
-                         "unit": "TOP/s", "frac": achieved / int8_peak,
-                         "peak_source": f"2 x sustained bf16 cuBLAS ({peaks['_source']})",
-                         "launches": int(g_n), "avg_launch_us": 1e3 * g_ms / max(g_n, 1), "traffic": GEMM_TRAFFIC_BYTES,
+            "roofline": {"kernel": "gemm_kernel<int8>", "bound": "tensor", "achieved": achieved, "peak": sustained2,
+                         "unit": "TOP/s", "frac": achieved / sustained2,
+                         "peak_source": f"2 x sustained bf16 cuBLAS ({peaks['_source']}; nominal int8:bf16 ratio)",
+                         "frac_of": frac_of, "peaks": {"2x_bf16_cublas_sustained": sustained2, "2x_bf16_cublas_burst": burst2,
+                                                       "datasheet_dense_int8_4500": DATASHEET_INT8_TOPS,
+                                                       "own_large_square_int8": own},
+                         "launches": int(g_n), "avg_launch_us": 1e3 * g_ms / max(g_n, 1),
+                         "kernel_ms_per_step": g_ms / args.steps, "bf16_kernel_ms_per_step": b_ms / args.steps,
+                         "traffic": GEMM_TRAFFIC_BYTES,
                          "traffic_source": "ncu dram bytes per launch, mean of the four GEMM launches (q/k/v grouped, o, ffn1, ffn2) of one block at 12288 tokens",
-                         "share_of_kernel_time": g_ms / max(g_ms + b_ms + o_ms, 1e-9), "share_of_step": g_ms / instrumented_ms,
-                         "how": "CUDA events around every launch in a second pass over the same steps"},
+                         "how": "the timed pass that gives `value`: every CTA folds %globaltimer after its wait for the "
+                                "previous kernel and at its end into the launch's slot; duration = last end - first start",
+                         "event_pass": {"int8_gemm_avg_launch_us": 1e3 * eg_ms / max(eg_n, 1),
+                                        "tops": eg_ops / (eg_ms * 1e-3) / 1e12 if eg_ms else None,
+                                        "share_of_kernel_time": eg_ms / max(eg_ms + eb_ms + eo_ms, 1e-9),
+                                        "step_ms": instrumented_ms,
+                                        "how": "one extra step with CUDA events around every launch (launches serialised)"}},
             "sweep": {"gbs": sweep_gbs, "ms": sweep_ms, "bytes": sweep_bytes, "hbm_peak_gbs": peaks["hbm_gbs"],
-                      "frac": sweep_gbs / peaks["hbm_gbs"], "peak_source": peaks["_source"]},
+                      "frac": sweep_gbs / peaks["hbm_gbs"], "peak_source": peaks["_source"],
+                      "sustained": {"calls": n_long, "gbs": sweep_long_gbs, "ms": sweep_long_ms, "sm_mhz": sweep_clock,
+                                    "hbm_frac": hbm_frac_long, "alu_frac": alu_frac,
+                                    "alu_peak_lane_ops_per_s": alu_peak, "lane_ops_per_element": 28,
+                                    "binds": "alu" if alu_frac > hbm_frac_long else "hbm"}},
             "search": search,
             "gemm_bf16": {"tflops": (b_ops / (b_ms * 1e-3) / 1e12) if b_ms else None, "launches": int(b_n)},
+            "workloads": workloads,
         }
         if not args.no_cpu_baseline and world == 1:
             te, ts, elems = oracle_sample(w, 768, 6)
@@ -387,6 +535,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used when profiling)")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the short legs of the other four workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

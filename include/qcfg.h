@@ -101,13 +101,19 @@ int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled);
  * one kernel.  Results are bit-identical either way.                                        */
 int qcfg_set_grouping(qcfg_ctx* ctx, int enabled);
 
-/* Per-launch timing of the GEMM kernel with CUDA events recorded on the launching stream
- * (off by default; a few microseconds of host time per launch when on).  kernel_class 0 is
- * the int8 GEMM, 1 the bf16 GEMM, 2 every other kernel of the library (except the sweep's
- * finalize step).  qcfg_profile_read waits for the recorded launches, then
- * returns the summed kernel time (ms), the number of launches and the summed algorithmic
- * operations (2*m*n*k per launch) since the last reset.  Outputs may be NULL.            */
-int qcfg_profile_enable(qcfg_ctx* ctx, int enabled);
+/* Per-launch timing, off by default.  Mode 1: CUDA events recorded around every launch on the
+ * launching stream (a few microseconds of host time per launch; the event records keep
+ * consecutive launches from overlapping, so a run in this mode is slower than an untimed one).
+ * kernel_class 0 is the int8 GEMM, 1 the bf16 GEMM, 2 every other kernel of the library (except
+ * the sweep's finalize step).  Mode 2: the GEMM kernels time themselves -- every CTA folds its
+ * %globaltimer reading after the wait for the previous kernel and at its end into the launch's
+ * slot of a ring in device memory (two atomics per CTA), so the duration of a launch is the span
+ * from its first CTA's start to its last CTA's end, measured inside an otherwise untouched run;
+ * classes 0 and 1 only, at most 65536 launches between two reads (later ones are not timed).
+ * qcfg_profile_read waits for the recorded launches (mode 2: for the device), then returns the
+ * summed kernel time (ms), the number of launches and the summed algorithmic operations
+ * (2*m*n*k per launch) since the last reset.  Outputs may be NULL.                          */
+int qcfg_profile_enable(qcfg_ctx* ctx, int mode);
 int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* launches, double* ops,
                       int reset);
 

@@ -162,8 +162,9 @@ class Context:
     def set_pair_tiles(self, enabled: bool):
         self._check(self.lib.qcfg_set_pair_tiles(self.h, int(enabled)))
 
-    def profile_enable(self, enabled: bool):
-        self._check(self.lib.qcfg_profile_enable(self.h, int(enabled)))
+    def profile_enable(self, mode):
+        """0 off, 1 CUDA events around every launch, 2 in-kernel time stamps of the GEMM launches."""
+        self._check(self.lib.qcfg_profile_enable(self.h, int(mode)))
 
     def profile_read(self, kernel_class: int, reset: bool = True):
         ms, n, ops = C.c_double(), C.c_int64(), C.c_double()

@@ -35,9 +35,46 @@ struct Ctx {
   size_t ev_used = 0;               // pairs in flight
   double prof_ms[3] = {0, 0, 0}, prof_ops[3] = {0, 0, 0};
   int64_t prof_n[3] = {0, 0, 0};
+  // in-kernel time stamps (profile mode 2): ring of {earliest start, latest end} pairs
+  unsigned long long* stamp_dev = nullptr;
+  std::vector<unsigned long long> stamp_host;   // the ring's initial pattern, then its read-back
+  std::vector<int> stamp_cls;
+  std::vector<double> stamp_ops;
+  size_t stamp_used = 0;
+  int64_t stamp_dropped = 0;
 };
 
 constexpr size_t kProfPairs = 8192;
+constexpr size_t kStampSlots = 65536;
+
+static int stamp_reset(Ctx* ctx) {
+  for (size_t i = 0; i < kStampSlots; ++i) { ctx->stamp_host[2 * i] = ~0ull; ctx->stamp_host[2 * i + 1] = 0ull; }
+  ctx->stamp_used = 0;
+  return check_cuda(ctx, cudaMemcpy(ctx->stamp_dev, ctx->stamp_host.data(), kStampSlots * 16, cudaMemcpyHostToDevice), "stamp ring reset");
+}
+// Waits for the device, folds the stamped launches into the per-class sums and clears the ring.
+static int stamp_drain(Ctx* ctx) {
+  if (!ctx->stamp_dev || ctx->stamp_used == 0) return QCFG_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(ctx->stamp_host.data(), ctx->stamp_dev, ctx->stamp_used * 16, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "stamp ring read");
+  for (size_t i = 0; i < ctx->stamp_used; ++i) {
+    const unsigned long long t0 = ctx->stamp_host[2 * i], t1 = ctx->stamp_host[2 * i + 1];
+    if (t1 <= t0) continue;                       // the launch did not run
+    const int c = ctx->stamp_cls[i];
+    ctx->prof_ms[c] += (double)(t1 - t0) * 1e-6;
+    ctx->prof_ops[c] += ctx->stamp_ops[i];
+    ctx->prof_n[c] += 1;
+  }
+  return stamp_reset(ctx);
+}
+unsigned long long* prof_stamp(Ctx* ctx, int cls, double ops) {
+  if (ctx->prof != 2) return nullptr;
+  if (ctx->stamp_used == kStampSlots) { ctx->stamp_dropped++; return nullptr; }
+  ctx->stamp_cls[ctx->stamp_used] = cls;
+  ctx->stamp_ops[ctx->stamp_used] = ops;
+  return ctx->stamp_dev + 2 * ctx->stamp_used++;
+}
 
 static void prof_drain(Ctx* ctx) {
   if (ctx->ev_used == 0) return;
@@ -52,13 +89,13 @@ static void prof_drain(Ctx* ctx) {
   ctx->ev_used = 0;
 }
 void prof_begin(Ctx* ctx, int cls, cudaStream_t st) {
-  if (!ctx->prof) return;
+  if (ctx->prof != 1) return;
   if (ctx->ev_used == kProfPairs) prof_drain(ctx);
   ctx->ev_cls[ctx->ev_used] = cls;
   cudaEventRecord(ctx->ev[2 * ctx->ev_used], st);
 }
 void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st) {
-  if (!ctx->prof) return;
+  if (ctx->prof != 1) return;
   cudaEventRecord(ctx->ev[2 * ctx->ev_used + 1], st);
   ctx->prof_ops[cls] += ops;
   ctx->ev_used += 1;
@@ -447,6 +484,7 @@ int qcfg_destroy(qcfg_ctx* ctx) {
   cudaDeviceSynchronize();
   for (auto& e : ctx->c.ev) cudaEventDestroy(e);
   if (ctx->c.scratch_buf) cudaFree(ctx->c.scratch_buf);
+  if (ctx->c.stamp_dev) cudaFree(ctx->c.stamp_dev);
   if (ctx->c.err_dev) cudaFree(ctx->c.err_dev);
   delete ctx;
   return QCFG_OK;
@@ -479,20 +517,31 @@ int64_t qcfg_launch_count(qcfg_ctx* ctx) { return ctx ? ctx->c.launches : 0; }
 int qcfg_profile_enable(qcfg_ctx* ctx, int enabled) {
   if (!ctx) return QCFG_EINVAL;
   Ctx* c = &ctx->c;
-  if (enabled && c->ev.empty()) {
+  if (enabled < 0 || enabled > 2) return set_error(c, QCFG_EINVAL, "profile: mode must be 0, 1 or 2");
+  if (enabled == 1 && c->ev.empty()) {
     c->ev.resize(2 * kProfPairs);
     c->ev_cls.resize(kProfPairs);
     for (auto& e : c->ev)
       if (cudaEventCreate(&e) != cudaSuccess) return set_error(c, QCFG_ECUDA, "profile: event creation failed");
   }
-  if (!enabled) prof_drain(c);
-  c->prof = enabled ? 1 : 0;
+  if (enabled == 2 && !c->stamp_dev) {
+    if (cudaMalloc(&c->stamp_dev, kStampSlots * 16) != cudaSuccess) { cudaGetLastError(); return set_error(c, QCFG_ENOMEM, "profile: stamp ring"); }
+    c->stamp_host.resize(2 * kStampSlots);
+    c->stamp_cls.resize(kStampSlots);
+    c->stamp_ops.resize(kStampSlots);
+    const int rc = stamp_reset(c);
+    if (rc) return rc;
+  }
+  if (c->prof == 1 && enabled != 1) prof_drain(c);
+  if (c->prof == 2 && enabled != 2) { const int rc = stamp_drain(c); if (rc) return rc; }
+  c->prof = enabled;
   return QCFG_OK;
 }
 int qcfg_profile_read(qcfg_ctx* ctx, int kernel_class, double* ms, int64_t* launches, double* ops, int reset) {
   if (!ctx || kernel_class < 0 || kernel_class > 2) return QCFG_EINVAL;
   Ctx* c = &ctx->c;
   prof_drain(c);
+  { const int rc = stamp_drain(c); if (rc) return rc; }
   if (ms) *ms = c->prof_ms[kernel_class];
   if (launches) *launches = c->prof_n[kernel_class];
   if (ops) *ops = c->prof_ops[kernel_class];

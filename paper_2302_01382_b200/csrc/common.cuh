@@ -31,6 +31,9 @@ bool sweep_tables_cached(Ctx* ctx, const void* dev_base, cudaStream_t st, const 
 // optional per-launch timing of one kernel class (0 = int8 GEMM, 1 = bf16 GEMM) with CUDA events
 void prof_begin(Ctx* ctx, int cls, cudaStream_t st);
 void prof_end(Ctx* ctx, int cls, double ops, cudaStream_t st);
+// in-kernel time stamps (profile mode 2): a device slot of two 64-bit words the launch's CTAs
+// fold their start and end times into, or nullptr when the mode is off or the ring is full
+unsigned long long* prof_stamp(Ctx* ctx, int cls, double ops);
 
 // ----- elementwise.cu -----------------------------------------------------------------
 int launch_absmax(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t ld,

@@ -33,6 +33,7 @@ constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;         // columns per accumulator buffer
 constexpr int kMaxStages = 8;
 constexpr int kSmemHeader = 1024;     // barriers and bookkeeping
+constexpr int kCsBytes = kEpiWarps * 64 * 4;   // per epilogue warp: rescale factors of its 64 columns
 constexpr int kSmemMax = 232448;      // 227 KB
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
@@ -50,11 +51,14 @@ struct OutDesc {
 // column tiles are numbered one after the other, so the persistent CTAs work through all of them
 // and only the first tile's main loop and the last tile's epilogue stay unoverlapped.
 constexpr int kMaxGroups = 3;
-struct GroupMaps { CUtensorMap a, b, om[kNumOuts]; };
+struct GroupMaps { CUtensorMap a, b, om[kNumOuts], fast; };   // fast: the output of a group served by a fast epilogue body
 struct AllMaps { GroupMaps g[kMaxGroups]; };
 // Epilogue bodies.  The general one handles any combination of outputs with run-time branches; the
 // two common combinations have straight-line bodies (same arithmetic, same order).
 enum : int32_t { EPI_GENERAL = 0, EPI_CODES1 = 1, EPI_Y = 2 };
+// Fast bodies (256-column tiles only): EPI_CODES1 writes each warp's 32 x 64 int8 block with one
+// TMA store (64-byte rows, 64B swizzle), EPI_Y each 32 x 32 fp32 block with one (128-byte rows,
+// 128B swizzle).
 struct GroupDesc {
   int32_t n, tn_begin;        // columns; first column-tile index of the group in the launch's numbering
   int32_t act;
@@ -71,6 +75,7 @@ struct GemmParams {
   uint32_t idesc;
   GroupDesc grp[kMaxGroups];  // unused groups have tn_begin = INT32_MAX
   unsigned* err;
+  unsigned long long* stamp;  // optional [2]: earliest start / latest end of the launch's CTAs (%globaltimer, ns)
 };
 
 // ---------------------------------------------------------------------------- PTX wrappers
@@ -230,6 +235,14 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&v)[32
         "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptors used by the MMA issuer: K-major tile of 128-byte rows, 128B
@@ -337,76 +350,120 @@ __device__ __forceinline__ void store_piece(const OutDesc& o, const CUtensorMap*
   }
 }
 
-// Rescale (and activate) one chunk: y[i] = act(acc[i] * cs[col i]); lane i holds the scale of column i.
+// ---- fast epilogue bodies -------------------------------------------------------------------
+// Two values at a time with packed fp32 instructions (same roundings as the scalar forms: each
+// half is an independent round-to-nearest operation).
+__device__ __forceinline__ float2 gelu_tanh2(float2 y) {
+  const float2 c1 = make_float2(-2.302208198f, -2.302208198f), c3 = make_float2(-0.1029432396f, -0.1029432396f);
+  const float2 y2 = __fmul2_rn(y, y);
+  const float2 t = __fmul2_rn(y, __ffma2_rn(c3, y2, c1));
+  float2 e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(t.x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(t.y));
+  const float2 d = __fadd2_rn(e, make_float2(1.0f, 1.0f));
+  float2 r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r.x) : "f"(d.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r.y) : "f"(d.y));
+  return __fmul2_rn(y, r);
+}
+// Rescaled and activated values of 16 accumulator columns of one row.  cs points to the 16
+// rescale factors of these columns in shared memory (every lane reads the same addresses).
 template <bool BF16>
-__device__ __forceinline__ void chunk_values(float (&y)[32], const uint32_t (&v)[32], float cs_lane, int act) {
+__device__ __forceinline__ void sub_values(float2 (&y)[8], const uint32_t (&v)[16], const float* cs, int act) {
   if (BF16) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(v[i]);
+    for (int i = 0; i < 8; ++i) y[i] = make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
   } else {
 #pragma unroll
-    for (int i = 0; i < 32; ++i)
-      y[i] = __fmul_rn((float)(int32_t)v[i], __shfl_sync(0xffffffffu, cs_lane, i));
+    for (int q = 0; q < 4; ++q) {
+      const float4 c = *reinterpret_cast<const float4*>(cs + 4 * q);
+      y[2 * q] = __fmul2_rn(make_float2((float)(int32_t)v[4 * q], (float)(int32_t)v[4 * q + 1]), make_float2(c.x, c.y));
+      y[2 * q + 1] = __fmul2_rn(make_float2((float)(int32_t)v[4 * q + 2], (float)(int32_t)v[4 * q + 3]), make_float2(c.z, c.w));
+    }
   }
   if (act == QCFG_ACT_RELU) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) y[i] = fmaxf(y[i], 0.0f);
+    for (int i = 0; i < 8; ++i) y[i] = make_float2(fmaxf(y[i].x, 0.0f), fmaxf(y[i].y, 0.0f));
   } else if (act == QCFG_ACT_GELU_TANH) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) y[i] = gelu_tanh(y[i]);
+    for (int i = 0; i < 8; ++i) y[i] = gelu_tanh2(y[i]);
   }
 }
-
-// EPI_CODES1: the only output is one int8 code matrix (slot 0) written by TMA; no shortcut.
-template <bool BF16>
-__device__ __forceinline__ void epilogue_chunk_codes1(const GroupDesc& p, const CUtensorMap* om, int m, uint32_t epi_bytes,
-                                                      const uint32_t (&v)[32], float cs_lane, int row0, int col0,
-                                                      uint32_t stage, uint32_t& cursor, int lane) {
-  if (p.n - col0 <= 0 || row0 >= m) return;        // warp-uniform: the piece lies outside the matrix
-  float y[32];
-  chunk_values<BF16>(y, v, cs_lane, p.act);
-  const float inv = p.outs[2].inv_scale, qmax = p.outs[2].qmax;
-  uint32_t w[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-    w[i] = pack4(code_word(y[4 * i], inv, qmax), code_word(y[4 * i + 1], inv, qmax),
-                 code_word(y[4 * i + 2], inv, qmax), code_word(y[4 * i + 3], inv, qmax));
-  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-  __syncwarp();
-  const uint32_t base = stage + (cursor & 1u) * (epi_bytes >> 1);
-  ++cursor;
-  st_shared_v4(base + lane * 32, w[0], w[1], w[2], w[3]);
-  st_shared_v4(base + lane * 32 + 16, w[4], w[5], w[6], w[7]);
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncwarp();
-  if (lane == 0) tma_store_2d(&om[2], base, col0, row0);
+// int8 codes of Eq. 1 for two values, each in the low byte of its word
+__device__ __forceinline__ float2 code_words2(float2 y, float2 inv2, float qmax) {
+  const float2 t = __fmul2_rn(y, inv2);
+  float2 c;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c.x) : "f"(t.x), "f"(qmax));
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(c.y) : "f"(t.y), "f"(qmax));
+  return __fadd2_rn(c, make_float2(12582912.0f, 12582912.0f));
 }
 
-// EPI_Y: the only output is the fp32 matrix written by TMA (two 16-column pieces); no shortcut.
-template <bool BF16>
-__device__ __forceinline__ void epilogue_chunk_y(const GroupDesc& p, const CUtensorMap* om, int m, uint32_t epi_bytes,
-                                                 const uint32_t (&v)[32], float cs_lane, int row0, int col0,
-                                                 uint32_t stage, uint32_t& cursor, int lane) {
-  const int ncols = p.n - col0;
-  if (ncols <= 0 || row0 >= m) return;
-  float y[32];
-  chunk_values<BF16>(y, v, cs_lane, p.act);
+// One warp's share of a 256-column tile (32 rows x 64 columns) in four pieces of 16 columns.
+// The accumulator load of the next piece is in flight while the current one is processed; the
+// accumulator buffer is released as soon as the last piece sits in registers.
+// CODES: one int8 matrix, the warp's 32 x 64 block staged in 64-byte rows (64B swizzle) and
+// written by one TMA store.  Otherwise the fp32 matrix, each 32 x 32 block staged in 128-byte
+// rows (128B swizzle), one TMA store per block; the single staging slot is reused once the
+// previous store has read it.
+template <bool BF16, bool PAIR, bool CODES>
+__device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUtensorMap* fmap, uint32_t tbase,
+                                                   const float* cs, uint32_t stage, int row0, int col0, int lane,
+                                                   uint32_t tempty_bar) {
+  const int act = G.act;
+  const float qmax = G.outs[2].qmax;
+  const float2 inv2 = make_float2(G.outs[2].inv_scale, G.outs[2].inv_scale);
+  uint32_t va[16], vb[16];
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the slot's last store was a tile ago
+  __syncwarp();
+  tmem_ld16_issue(tbase, va);
+  auto piece = [&](const uint32_t (&v)[16], int s) {
+    float2 y[8];
+    sub_values<BF16>(y, v, cs + 16 * s, act);
+    if (CODES) {
+      uint32_t w[4];
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    if (h == 1 && ncols <= 16) break;
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-    __syncwarp();
-    const uint32_t base = stage + (cursor & 1u) * (epi_bytes >> 1);
-    ++cursor;
+      for (int j = 0; j < 4; ++j) {
+        const float2 a = code_words2(y[2 * j], inv2, qmax), b = code_words2(y[2 * j + 1], inv2, qmax);
+        w[j] = pack4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(b.x), __float_as_uint(b.y));
+      }
+      st_shared_v4(stage + lane * 64 + ((s ^ ((lane >> 1) & 3)) << 4), w[0], w[1], w[2], w[3]);
+    } else {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int js = j ^ ((lane >> 1) & 3);
-      st_shared_v4(base + lane * 64 + js * 16, __float_as_uint(y[16 * h + 4 * j]), __float_as_uint(y[16 * h + 4 * j + 1]),
-                   __float_as_uint(y[16 * h + 4 * j + 2]), __float_as_uint(y[16 * h + 4 * j + 3]));
+      for (int j = 0; j < 4; ++j) {
+        const int p16 = 4 * (s & 1) + j;
+        st_shared_v4(stage + lane * 128 + ((p16 ^ (lane & 7)) << 4), __float_as_uint(y[2 * j].x), __float_as_uint(y[2 * j].y),
+                     __float_as_uint(y[2 * j + 1].x), __float_as_uint(y[2 * j + 1].y));
+      }
     }
+  };
+#pragma unroll 1
+  for (int h = 0; h < 2; ++h) {
+    tmem_ld_wait();
+    tmem_ld16_issue(tbase + 32 * h + 16, vb);
+    if (!CODES && h == 1) {   // the first block's store must have read the slot before it is refilled
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();
+    }
+    piece(va, 2 * h);
+    tmem_ld_wait();
+    if (h == 0) {
+      tmem_ld16_issue(tbase + 32, va);
+    } else {          // every column of this warp is in registers: the accumulator buffer is free
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
+    }
+    piece(vb, 2 * h + 1);
+    if (!CODES) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0 && col0 + 32 * h < G.n) tma_store_2d(fmap, stage, col0 + 32 * h, row0);
+    }
+  }
+  if (CODES) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0) tma_store_2d(&om[1], base, col0 + 16 * h, row0);
+    if (lane == 0) tma_store_2d(fmap, stage, col0, row0);
   }
 }
 
@@ -495,7 +552,8 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);           // full[8] empty[8] tfull[2] tempty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
-  uint8_t* epi_stage = smem + kSmemHeader;                       // kEpiWarps x epi_bytes, 1024-aligned
+  float* cs_all = reinterpret_cast<float*>(smem + kSmemHeader);  // kEpiWarps x 64 rescale factors
+  uint8_t* epi_stage = smem + kSmemHeader + kCsBytes;            // kEpiWarps x epi_bytes, 1024-aligned
   uint8_t* stage_base = epi_stage + kEpiWarps * p.epi_bytes;
 
   const int warp = threadIdx.x >> 5;
@@ -517,6 +575,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   auto group_of = [&](int tn) -> int {
     return GROUPED ? (int)(tn >= p.grp[1].tn_begin) + (int)(tn >= p.grp[2].tn_begin) : 0;
   };
+  auto tile_in_group = [&](int tn, int g) -> int { return GROUPED ? tn - p.grp[g].tn_begin : tn; };
   // Tiles are numbered with the row-tile index fastest.  Each role walks its tiles by adding the
   // stride split into (row tiles, column tiles) once here: a division per tile would sit on the
   // epilogue's and the producer's path.
@@ -541,7 +600,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
     const int g = group_of(ld_tn);
     if (GROUPED) { ld_map_a = &maps.g[g].a; ld_map_b = &maps.g[g].b; }
     ld_ya = ld_tm * rows_per_tile + rank * BM;
-    ld_yb = (ld_tn - (GROUPED ? p.grp[g].tn_begin : 0)) * p.bn + rank * b_rows;
+    ld_yb = tile_in_group(ld_tn, g) * p.bn + rank * b_rows;
   };
   set_tile_coords();
   const bool elected = elect_one();    // the lane of a converged warp that issues TMA / MMA instructions
@@ -592,6 +651,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   // Everything above touches no global memory, so under programmatic dependent launch it
   // overlaps the tail of the previous kernel in the stream; from here on its results are needed.
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (p.stamp && threadIdx.x == 32) atomicMin(p.stamp, (unsigned long long)global_timer());
   if (warp == 0) {
     // the ring is empty: fill it before the block-wide barrier so the first tiles are in flight
     for (int i = 0; i < p.stages && ld_tile < num_tiles; ++i) issue_load();
@@ -674,7 +734,9 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
     const int c_begin = colgrp * cpg;
     const int c_end = c_begin < chunks ? c_begin + cpg : c_begin;
     const uint32_t stage = smem_u32(epi_stage + ew * p.epi_bytes);
+    float* cs_tab = cs_all + ew * 64;
     uint32_t cursor = 0;
+    bool prev_fast = false;
     bool ok = true;
     int t = 0;
     // Weight scales of this warp's chunks, one column per lane and chunk.  They are fetched one
@@ -683,9 +745,10 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
     auto load_scales = [&](int tile, int tile_tn, float (&w)[2]) {
       w[0] = 0.f; w[1] = 0.f;
       if (BF16 || tile >= num_tiles) return;
-      const GroupDesc& G = p.grp[group_of(tile_tn)];
+      const int gi = group_of(tile_tn);
+      const GroupDesc& G = p.grp[gi];
       if (!G.need_y) return;
-      const int cb = (tile_tn - (GROUPED ? G.tn_begin : 0)) * p.bn + c_begin * 32;
+      const int cb = tile_in_group(tile_tn, gi) * p.bn + c_begin * 32;
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int col = cb + j * 32 + lane;
@@ -700,7 +763,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
       const int row0 = tm * rows_per_tile + rank * BM + quad * 32;
       const int g = group_of(tn);
       const GroupDesc& G = p.grp[g];
-      const int col_base = (tn - (GROUPED ? G.tn_begin : 0)) * p.bn + c_begin * 32;
+      const int col_base = tile_in_group(tn, g) * p.bn + c_begin * 32;
       const float cs[2] = {__fmul_rn(G.scale_x, sw_next[0]), __fmul_rn(G.scale_x, sw_next[1])};
       int tm_next = tm + step_tm, tn_next = tn + step_tn;
       if (tm_next >= p.tiles_m) { tm_next -= p.tiles_m; ++tn_next; }
@@ -710,28 +773,48 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
       const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * kAccCols + c_begin * 32);
       const int nch = c_end - c_begin;           // 0, 1 or 2
       const int64_t row = (int64_t)row0 + lane;
-      uint32_t v[32];
-      // one copy of the chunk code, looped: keeps the instruction footprint small
-#pragma unroll 1
-      for (int c = 0; c < nch; ++c) {
-        tmem_ld32_issue(tbase + 32 * c, v);
-        tmem_ld_wait();
-        if (c == nch - 1) {   // the accumulator buffer is free again once this warp's columns sit in registers
-          tc_fence_before();
+      const uint32_t tempty_bar = tempty0 + 8 * a;
+      if (G.mode != EPI_GENERAL) {
+        // fast bodies: 256-column tiles, so this warp owns 64 columns starting at col_base
+        if (row0 >= p.m || col_base >= G.n) {
           __syncwarp();
-          if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
+          if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
+        } else {
+          if (!BF16) {   // rescale factors of the 64 columns, read back by every lane
+            cs_tab[lane] = cs[0];
+            cs_tab[32 + lane] = cs[1];
+            __syncwarp();
+          }
+          if (G.mode == EPI_CODES1)
+            epilogue_tile_fast<BF16, PAIR, true>(G, &maps.g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar);
+          else
+            epilogue_tile_fast<BF16, PAIR, false>(G, &maps.g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar);
         }
-        const float csl = c ? cs[1] : cs[0];
-        if (G.mode == EPI_CODES1)
-          epilogue_chunk_codes1<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row0, col_base + 32 * c, stage, cursor, lane);
-        else if (G.mode == EPI_Y)
-          epilogue_chunk_y<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row0, col_base + 32 * c, stage, cursor, lane);
-        else
+        prev_fast = true;
+      } else {
+        if (prev_fast) {    // a fast body's last store reads the whole staging buffer: let it finish
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          __syncwarp();
+          prev_fast = false;
+        }
+        uint32_t v[32];
+        // one copy of the chunk code, looped: keeps the instruction footprint small
+#pragma unroll 1
+        for (int c = 0; c < nch; ++c) {
+          tmem_ld32_issue(tbase + 32 * c, v);
+          tmem_ld_wait();
+          if (c == nch - 1) {   // the accumulator buffer is free again once this warp's columns sit in registers
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
+          }
+          const float csl = c ? cs[1] : cs[0];
           epilogue_chunk<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
-      }
-      if (nch == 0) {
-        __syncwarp();
-        if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty0 + 8 * a); else mbar_arrive(tempty0 + 8 * a); }
+        }
+        if (nch == 0) {
+          __syncwarp();
+          if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
+        }
       }
       tm = tm_next; tn = tn_next;
     }
@@ -741,6 +824,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
 
   tc_fence_before();
   __syncthreads();
+  if (p.stamp && threadIdx.x == 32) atomicMax(p.stamp + 1, (unsigned long long)global_timer());
   if (PAIR) cluster_sync_all();     // the peer no longer signals this CTA's barriers nor uses its TMEM
   if (warp == 1) {
     tc_fence_after();
@@ -787,6 +871,23 @@ bool make_out_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(map, dt, 2, o.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         esz == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Tensor map of the output a fast epilogue body writes: 32-row boxes of 64 int8 columns (64B
+// swizzle) or of 32 fp32 columns (128B swizzle).
+bool make_fast_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
+  const bool codes = o.kind == 1;
+  const int esz = codes ? 1 : 4;
+  if (((uintptr_t)o.ptr & 15) || ((o.ld * esz) & 15)) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)m};
+  cuuint64_t strides[1] = {(cuuint64_t)(o.ld * esz)};
+  cuuint32_t box[2] = {codes ? 64u : 32u, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, codes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, o.ptr, dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        codes ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -903,9 +1004,9 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
     // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
     for (int j = 0; j < kNumOuts; ++j) if (G.outs[j].kind >= 2 && G.outs[j].tma) wide = true;
     G.mode = EPI_GENERAL;
-    if (!G.residual && !G.outs[0].kind && !G.outs[3].kind && !G.outs[4].kind) {
-      if (!G.outs[1].kind && G.outs[2].kind == 1 && G.outs[2].tma) G.mode = EPI_CODES1;
-      else if (G.outs[1].kind && G.outs[1].tma && !G.outs[2].kind) G.mode = EPI_Y;
+    if (bn == 256 && !G.residual && !G.outs[0].kind && !G.outs[3].kind && !G.outs[4].kind) {
+      if (!G.outs[1].kind && G.outs[2].kind == 1 && make_fast_map(&maps.g[i].fast, G.outs[2], g.m, g.n)) G.mode = EPI_CODES1;
+      else if (G.outs[1].kind && !G.outs[2].kind && make_fast_map(&maps.g[i].fast, G.outs[1], g.m, g.n)) { G.mode = EPI_Y; wide = true; }
     }
     int rc = make_map(ctx, &maps.g[i].a, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
     if (rc == QCFG_OK) rc = make_map(ctx, &maps.g[i].b, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
@@ -914,7 +1015,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
   }
   p.tiles_n = tn_total;
   p.epi_bytes = wide ? 4096 : 2048;
-  int stages = (kSmemMax - kSmemHeader - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
+  int stages = (kSmemMax - kSmemHeader - kCsBytes - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   p.stages = stages;
 
@@ -941,7 +1042,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
     grid = 2 * (*cached);
     if (grid > 2 * num_tiles) grid = 2 * num_tiles;
   } else if (grid > num_tiles) grid = num_tiles;
-  const size_t smem = (size_t)kSmemHeader + 1024 + (size_t)kEpiWarps * p.epi_bytes + (size_t)stages * stage_bytes;
+  const size_t smem = (size_t)kSmemHeader + kCsBytes + 1024 + (size_t)kEpiWarps * p.epi_bytes + (size_t)stages * stage_bytes;
   // Programmatic dependent launch: the kernel's prologue (barrier set-up, TMEM allocation) may
   // start while the previous kernel in the stream drains; it waits (griddepcontrol.wait) before
   // touching global memory.
@@ -962,6 +1063,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       gemm_kernel<false, false, false>, gemm_kernel<false, false, true>, gemm_kernel<false, true, false>, gemm_kernel<false, true, true>,
       gemm_kernel<true, false, false>,  gemm_kernel<true, false, true>,  gemm_kernel<true, true, false>,  gemm_kernel<true, true, true>};
   const Kern kern = kernels[(g0.is_bf16 ? 4 : 0) + (pair ? 2 : 0) + (count > 1 ? 1 : 0)];
+  p.stamp = prof_stamp(ctx, g0.is_bf16 ? 1 : 0, ops);
   prof_begin(ctx, g0.is_bf16 ? 1 : 0, st);
   const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, maps, p);
   prof_end(ctx, g0.is_bf16 ? 1 : 0, ops, st);
