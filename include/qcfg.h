@@ -160,15 +160,14 @@ int qcfg_quant_error_sweep(qcfg_ctx* ctx, const float* const* w_dev, const int64
  * device-wide synchronisation of cudaMalloc/cudaFree is not acceptable.  (The paper has no
  * counterpart; this is a deployment variant of qcfg_quant_error_sweep.)  Arguments, outputs and
  * results are those of qcfg_quant_error_sweep.  Differences:
- *   - Its scratch memory (block partial sums and descriptor tables) is a fixed array inside
- *     the library image, about 1.05 MiB on every GPU that loads the library, held until the
- *     process exits.  The call itself performs no cudaMalloc, cudaFree or other device allocation.
- *   - Limits per call: at most 1024 tensors and at most 16384 work items.  A work item is a
- *     run of whole rows of one tensor holding about total/(8 * SM count) elements, between
- *     8 Ki and 256 Ki, so the item limit is only reached by inputs beyond 4 Gi elements or with
- *     rows longer than 256 Ki elements in great number.  Anything larger returns QCFG_ENOMEM
- *     with a message and does nothing; split the tensors over several calls, one after the
- *     other.
+ *   - Its scratch memory (partial sums and work tables) is a fixed array inside the library
+ *     image, about 0.6 MiB on every GPU that loads the library, held until the process exits.
+ *     The call itself performs no cudaMalloc, cudaFree or other device allocation.
+ *   - Limits per call: at most 1024 tensors and at most 2^35 elements in total.  Anything larger
+ *     returns QCFG_ENOMEM with a message and does nothing; split the tensors over several calls,
+ *     one after the other.
+ *   - The work tables are copied to the device from host memory the context reuses on the next
+ *     call, so the call must not be recorded into a CUDA graph by stream capture.
  *   - ctx's device must be the current device (QCFG_ESTATE otherwise).  The first call on a
  *     device looks up the array's device address (cudaGetSymbolAddress) and keeps it; make
  *     that first call during start-up, before any stream capture begins.

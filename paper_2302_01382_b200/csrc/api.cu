@@ -28,6 +28,7 @@ struct Ctx {
   const void* sweep_base = nullptr;
   cudaStream_t sweep_stream = nullptr;
   std::vector<char> sweep_tables;
+  std::vector<char> host_buf;       // host-side planning tables
   // per-launch event timing (off by default)
   int prof = 0;
   std::vector<cudaEvent_t> ev;      // pairs: ev[2i] before, ev[2i+1] after
@@ -123,14 +124,22 @@ int check_cuda(Ctx* ctx, cudaError_t e, const char* what) {
 }
 bool sweep_tables_cached(Ctx* ctx, const void* dev_base, cudaStream_t st, const void* a, size_t na, const void* b, size_t nb) {
   if (ctx->sweep_base == dev_base && ctx->sweep_stream == st && ctx->sweep_tables.size() == na + nb &&
-      memcmp(ctx->sweep_tables.data(), a, na) == 0 && memcmp(ctx->sweep_tables.data() + na, b, nb) == 0)
+      memcmp(ctx->sweep_tables.data(), a, na) == 0 && (nb == 0 || memcmp(ctx->sweep_tables.data() + na, b, nb) == 0))
     return true;
   ctx->sweep_tables.resize(na + nb);
   memcpy(ctx->sweep_tables.data(), a, na);
-  memcpy(ctx->sweep_tables.data() + na, b, nb);
+  if (nb) memcpy(ctx->sweep_tables.data() + na, b, nb);
   ctx->sweep_base = dev_base;
   ctx->sweep_stream = st;
   return false;
+}
+void* host_scratch(Ctx* ctx, size_t bytes) {
+  try {
+    if (ctx->host_buf.size() < bytes) ctx->host_buf.resize(bytes);
+  } catch (...) {
+    return nullptr;
+  }
+  return ctx->host_buf.data();
 }
 void* scratch(Ctx* ctx, size_t bytes) {
   if (bytes <= ctx->scratch_bytes) return ctx->scratch_buf;

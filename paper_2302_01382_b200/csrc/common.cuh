@@ -25,6 +25,8 @@ int* pair_cluster_cache(Ctx* ctx);   // [2]: resident CTA pairs of the int8 / bf
 int device_of(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);
+// grows (never shrinks) a host buffer owned by the context; returns nullptr on failure
+void* host_scratch(Ctx* ctx, size_t bytes);
 // true when the same two host tables were the last ones uploaded to this scratch address on
 // this context in this stream (the caller may then skip the upload); records them otherwise
 bool sweep_tables_cached(Ctx* ctx, const void* dev_base, cudaStream_t st, const void* a, size_t na, const void* b, size_t nb);

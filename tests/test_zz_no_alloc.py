@@ -57,6 +57,30 @@ def test_static_sweep_matches_regular_sweep_on_two_calls_in_a_row():
         ctx.close()
 
 
+def test_static_sweep_matches_the_oracle_and_allocates_nothing():
+    """Against the CPU oracle (not only its sibling), and with the device's free memory unchanged
+    across a call once the outputs exist."""
+    import paper_2302_01382_b200 as q
+    from oracle import qcfg_oracle as orc
+    ctx = q.Context(0)
+    try:
+        tensors = _tensors(3, [(200, 768), (64, 3072), (33, 100)])
+        so, ao = orc.quant_error_sweep([t.cpu().numpy() for t in tensors])
+        sse = torch.empty((3, 7), dtype=torch.float64, device="cuda")
+        amax = torch.empty(3, dtype=torch.float32, device="cuda")
+        ctx.quant_error_sweep_static(tensors, q.PER_ROW, 2, 8, sse=sse, absmax=amax)      # first call: address look-up
+        ctx.check_sync()
+        free_before, _ = torch.cuda.mem_get_info()
+        ctx.quant_error_sweep_static(tensors, q.PER_ROW, 2, 8, sse=sse, absmax=amax)
+        ctx.check_sync()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
+        np.testing.assert_allclose(sse.cpu().numpy(), so, rtol=1e-5)
+        np.testing.assert_array_equal(amax.cpu().numpy(), ao)
+    finally:
+        ctx.close()
+
+
 def test_static_sweep_refuses_what_does_not_fit():
     import paper_2302_01382_b200 as q
     ctx = q.Context(0)
@@ -64,11 +88,11 @@ def test_static_sweep_refuses_what_does_not_fit():
         t = torch.zeros((8, 64), device="cuda")
         sse = torch.zeros((1, 7), dtype=torch.float64, device="cuda")
         amax = torch.zeros(1, device="cuda")
-        # a declared shape needing far more work items than the array holds: refused on the host,
-        # nothing is launched, outputs stay as they were
+        # a declared shape beyond the element limit of one call: refused on the host, nothing is
+        # launched, outputs stay as they were
         with pytest.raises(q.QcfgError) as e:
             ctx.quant_error_sweep_static([t], q.PER_ROW, 2, 8, sse=sse, absmax=amax, shapes=[(10 ** 9, 768)])
-        assert e.value.status == q.ENOMEM and "work items" in str(e.value)
+        assert e.value.status == q.ENOMEM and "2^35 elements" in str(e.value)
         many = [t] * 1025
         with pytest.raises(q.QcfgError) as e:
             ctx.quant_error_sweep_static(many, q.PER_ROW, 2, 8)
