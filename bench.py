@@ -462,6 +462,19 @@ def run_gpu(args):
         dt = time.perf_counter() - t0
         search = {"algorithm": "greedy", "bs": [8, 4], "target_fidelity": 0.9, "evals": int(n_s), "ms": 1e3 * dt,
                   "evals_per_s": n_s / dt, "layers_at_4_bit": int(sum(1 for b in bits_s if b == 4))}
+        # the same search with prefix reuse: every evaluation restarts at the first layer whose
+        # width changed (reported beside the full-recompute figures, never instead of them)
+        ctx.set_prefix_reuse(True)
+        l0 = ctx.launch_count()
+        t0 = time.perf_counter()
+        bits_r, vis_r, acc_r, n_r = job.model.search(q.SEARCH_GREEDY, rank_now, [8, 4], 0.9, job.x, w.m)
+        torch.cuda.synchronize()
+        dt_r = time.perf_counter() - t0
+        ctx.set_prefix_reuse(False)
+        search["prefix_reuse_evals_per_s"] = n_r / dt_r
+        search["prefix_reuse_ms"] = 1e3 * dt_r
+        search["prefix_reuse_launches"] = int(ctx.launch_count() - l0)
+        search["prefix_reuse_same_result"] = bool(bits_r == bits_s and vis_r == vis_s and acc_r == acc_s)
 
     # ---------------- the other four workloads
     workloads = None

@@ -101,6 +101,17 @@ int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled);
  * one kernel.  Results are bit-identical either way.                                        */
 int qcfg_set_grouping(qcfg_ctx* ctx, int enabled);
 
+/* Switches prefix reuse in model evaluations (default off).  On: qcfg_eval_config keeps every
+ * layer's buffers from the previous evaluation and, when it is called again with the same x_dev,
+ * the same m and no switch changed in between, recomputes only the layers whose bit width changed,
+ * the layers whose output the caller asks for, and everything that reads a recomputed layer; the
+ * other layers launch nothing.  This is what consecutive configurations of the searches allow:
+ * Algorithm 2 changes one layer per evaluation, Algorithm 1 a slice of the ordering.  The CALLER
+ * guarantees that the contents of x_dev did not change between such calls.  Results are
+ * bit-identical to a full evaluation.  qcfg_calibrate_model, qcfg_latency_table and
+ * qcfg_noise_sensitivity always run every layer.                                              */
+int qcfg_set_prefix_reuse(qcfg_ctx* ctx, int enabled);
+
 /* Per-launch timing, off by default.  Mode 1: CUDA events recorded around every launch on the
  * launching stream (a few microseconds of host time per launch; the event records keep
  * consecutive launches from overlapping, so a run in this mode is slower than an untimed one).
