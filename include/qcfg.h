@@ -302,6 +302,37 @@ int qcfg_search(qcfg_ctx* ctx, qcfg_model* model, int algorithm, const int32_t* 
                 uint8_t* bits_out, uint8_t* visited, double* accuracies, int32_t capacity,
                 int32_t* n_evals, void* stream);
 
+/* Scale adjustment (Section 3.1, second step of the scale estimation; Section 4 gives the
+ * learning rate 1e-5): after max calibration the quantization scales are adapted by
+ * backpropagation, the model's own parameters staying fixed.  The loss needs labels the library
+ * does not have: L = sum (y - y_ref)^2 / sum y_ref^2 on the LAST layer's fp32 output, y_ref being
+ * the output with every layer at 16 bit.  The rounding of Eq. 1 is differentiated straight through
+ * (derivative 1 inside the clip range, 0 outside).  All four kinds of scale of every layer that
+ * runs at an integer width under bits[] are adapted: the activation's scale and inv_scale (one pair
+ * per layer) and the weight's per output channel.  Each of `steps` steps is one forward, one
+ * backward (two bf16 tensor-core GEMMs per layer) and scale <- float(scale - lr * gradient) on the
+ * whole batch x_dev; losses_host (HOST, steps + 1 doubles, may be NULL) receives the loss before
+ * every step and after the last.  From then on qcfg_eval_config uses the adapted scales wherever a
+ * layer runs at the width it was adapted at; qcfg_calibrate_model and qcfg_model_reset_scales go
+ * back to max calibration.  Linear layers only (QCFG_ESHAPE for a convolutional table).
+ * Synchronises the stream several times per step.                                              */
+int qcfg_adjust_scales(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, const float* x_dev,
+                       int64_t m, int32_t steps, double lr, double* losses_host, void* stream);
+/* The gradients one step of qcfg_adjust_scales would use, at the model's current scales (HOST
+ * outputs, any may be NULL): d_scale_x[n_layers], d_inv_scale_x[n_layers] (0 for 16-bit layers);
+ * d_scale_w / d_inv_scale_w are HOST arrays of n_layers HOST pointers to n_out doubles each (a NULL
+ * entry skips the layer; 16-bit layers give zeros); *loss the loss.  Changes no scale.          */
+int qcfg_scale_gradients(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, const float* x_dev,
+                         int64_t m, double* d_scale_x, double* d_inv_scale_x,
+                         double* const* d_scale_w, double* const* d_inv_scale_w, double* loss,
+                         void* stream);
+/* The scales layer `layer` uses at `bits` (2..8) right now: the activation pair and, to HOST arrays
+ * of n_out floats, the weight's per-channel pairs.  Outputs may be NULL.                        */
+int qcfg_model_scales(qcfg_model* model, int32_t layer, int bits, float* scale_x,
+                      float* inv_scale_x, float* scale_w_host, float* inv_scale_w_host);
+/* Discards every adapted scale: all layers are back at their max-calibrated scales.             */
+int qcfg_model_reset_scales(qcfg_model* model);
+
 /* Parity taps for layer `layer` of the LAST qcfg_eval_config call (same stream order):
  * the int8 codes of its GEMM input (qx_dev, [rows x k_in] dense, or NULL), of its weight
  * (qw_dev, [n_out x k_in] dense, or NULL) and its raw int32 accumulators (acc_dev,

@@ -27,7 +27,8 @@ EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_selftest_wai
            "qcfg_set_fusion", "qcfg_set_pair_tiles", "qcfg_set_grouping", "qcfg_set_prefix_reuse", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
-           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_latency_table", "qcfg_config_cost", "qcfg_noise_sensitivity", "qcfg_search", "qcfg_debug_dump"]
+           "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_latency_table", "qcfg_config_cost", "qcfg_noise_sensitivity", "qcfg_search", "qcfg_adjust_scales", "qcfg_scale_gradients", "qcfg_model_scales",
+           "qcfg_model_reset_scales", "qcfg_debug_dump"]
 
 
 class QcfgError(RuntimeError):
@@ -86,6 +87,11 @@ def load_library() -> C.CDLL:
         "qcfg_search": [vp, vp, ci, C.POINTER(i32), C.POINTER(C.c_uint8), i32, C.c_double, vp, i64, C.POINTER(C.c_uint8),
                         C.POINTER(C.c_uint8), C.POINTER(C.c_double), i32, C.POINTER(i32), vp],
         "qcfg_noise_sensitivity": [vp, vp, vp, i64, C.POINTER(C.c_void_p), C.c_float, C.POINTER(C.c_double), vp],
+        "qcfg_adjust_scales": [vp, vp, C.POINTER(C.c_uint8), vp, i64, i32, C.c_double, C.POINTER(C.c_double), vp],
+        "qcfg_scale_gradients": [vp, vp, C.POINTER(C.c_uint8), vp, i64, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                 C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_double), vp],
+        "qcfg_model_scales": [vp, i32, ci, C.POINTER(f32), C.POINTER(f32), C.POINTER(f32), C.POINTER(f32)],
+        "qcfg_model_reset_scales": [vp],
         "qcfg_latency_table": [vp, vp, vp, i64, C.POINTER(C.c_uint8), i32, i32, C.POINTER(C.c_float), vp],
         "qcfg_config_cost": [vp, C.POINTER(C.c_uint8), C.POINTER(C.c_uint8), i32, C.POINTER(C.c_float), C.POINTER(C.c_double),
                              C.POINTER(C.c_double)],
@@ -333,6 +339,37 @@ class Model:
         out = (C.c_double * n)()
         self.ctx._check(self.ctx.lib.qcfg_noise_sensitivity(self.ctx.h, self.h, _ptr(x), m, ptrs, float(lam), out, _stream(stream)))
         return list(out)
+
+    def adjust_scales(self, bits, x: torch.Tensor, m: int, steps: int, lr: float = 1e-5, stream=None):
+        """Section 3.1's adjustment step: `steps` gradient steps on the scales.  Returns the losses (steps + 1)."""
+        n = len(self.layers)
+        b = (C.c_uint8 * n)(*[int(v) for v in bits])
+        losses = (C.c_double * (steps + 1))()
+        self.ctx._check(self.ctx.lib.qcfg_adjust_scales(self.ctx.h, self.h, b, _ptr(x), m, steps, float(lr), losses, _stream(stream)))
+        return list(losses)
+
+    def scale_gradients(self, bits, x: torch.Tensor, m: int, stream=None):
+        """(loss, d_scale_x, d_inv_scale_x, d_scale_w, d_inv_scale_w); the last two are lists of per-channel lists."""
+        n = len(self.layers)
+        b = (C.c_uint8 * n)(*[int(v) for v in bits])
+        dsx, dix, loss = (C.c_double * n)(), (C.c_double * n)(), C.c_double()
+        bufs_s = [(C.c_double * l.n_out)() for l in self.layers]
+        bufs_i = [(C.c_double * l.n_out)() for l in self.layers]
+        ps = (C.c_void_p * n)(*[C.addressof(a) for a in bufs_s])
+        pi = (C.c_void_p * n)(*[C.addressof(a) for a in bufs_i])
+        self.ctx._check(self.ctx.lib.qcfg_scale_gradients(self.ctx.h, self.h, b, _ptr(x), m, dsx, dix, ps, pi, C.byref(loss), _stream(stream)))
+        return loss.value, list(dsx), list(dix), [list(a) for a in bufs_s], [list(a) for a in bufs_i]
+
+    def scales(self, layer: int, bits: int):
+        """(scale_x, inv_scale_x, scale_w[n_out], inv_scale_w[n_out]) in use for `layer` at `bits`."""
+        n_out = self.layers[layer].n_out
+        sx, ix = C.c_float(), C.c_float()
+        sw, iw = (C.c_float * n_out)(), (C.c_float * n_out)()
+        self.ctx._check(self.ctx.lib.qcfg_model_scales(self.h, layer, bits, C.byref(sx), C.byref(ix), sw, iw))
+        return sx.value, ix.value, list(sw), list(iw)
+
+    def reset_scales(self):
+        self.ctx._check(self.ctx.lib.qcfg_model_reset_scales(self.h))
 
     def latency_table(self, x: torch.Tensor, m: int, bs, reps: int = 5, stream=None):
         """Mean milliseconds of every layer at every width of bs: list of n_layers rows of len(bs) floats."""

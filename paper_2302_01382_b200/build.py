@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libqcfg.so")
-SOURCES = ["api.cu", "elementwise.cu", "conv.cu", "sweep.cu", "gemm.cu"]
+SOURCES = ["api.cu", "elementwise.cu", "conv.cu", "sweep.cu", "gemm.cu", "adjust.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -180,7 +180,8 @@ struct WeightCodes {
   DevBuf codes;           // int8 or bf16 [n_out x ldk]
   DevBuf scale;           // fp32 [n_out] post-rounding scales (int only)
   DevBuf inv;             // fp32 [n_out] pre-rounding scales (int only)
-  bool ready = false;
+  bool ready = false;     // codes match the scales
+  bool adjusted = false;  // the scales no longer come from the calibrated maxima (scale adjustment)
 };
 
 struct LayerState {
@@ -189,6 +190,10 @@ struct LayerState {
   DevBuf w_absmax;                 // fp32 [n_out]
   WeightCodes wc[17];              // by bit width
   float act_absmax = 0.0f;         // calibrated max|input|
+  // activation scales after scale adjustment, by bit width (otherwise derived from act_absmax)
+  bool adj_act[17] = {false};
+  float adj_sx[17] = {0}, adj_ix[17] = {0};
+  DevBuf ylin, yact, gout, dsw, diw;   // scale adjustment: rescaled accumulators, activated output, dL/d(output), weight scale gradients
   std::vector<int> consumers;      // layers reading this layer's output as GEMM input
   bool feeds_residual = false;
   // per-evaluation state
@@ -214,6 +219,7 @@ struct Model {
   DevBuf act_absmax_dev;           // fp32 [n_layers], filled by calibration
   DevBuf search_ref, search_out, search_partial;   // buffers of the search drivers
   DevBuf noise_codes, noise_amax;                  // perturbed bf16 weights of one layer and its max|w|
+  DevBuf adj_gs, adj_gt, adj_qxt, adj_qwt, adj_dx, adj_dw, adj_colsum, adj_dscal;   // scale adjustment temporaries
   int64_t last_m = 0;
   // what the layers' buffers hold after the last evaluation (for prefix reuse)
   bool reuse_valid = false;
@@ -257,7 +263,7 @@ int ensure_weight_codes(Ctx* ctx, LayerState& S, int bits, cudaStream_t st) {
   } else {
     rc = W.scale.ensure(ctx, (size_t)n * 4);
     if (!rc) rc = W.inv.ensure(ctx, (size_t)n * 4);
-    if (!rc) rc = launch_scales(ctx, (const float*)S.w_absmax.p, n, bits, (float*)W.scale.p, (float*)W.inv.p, st);
+    if (!rc && !W.adjusted) rc = launch_scales(ctx, (const float*)S.w_absmax.p, n, bits, (float*)W.scale.p, (float*)W.inv.p, st);
     if (!rc) rc = launch_quantize(ctx, S.d.w_dev, n, k, k, (const float*)W.inv.p, 1.0f, QCFG_PER_ROW, bits, W.codes.p, S.ldk, st);
   }
   if (rc) return rc;
@@ -273,7 +279,13 @@ inline void host_scales(float A, int bits, float* scale, float* inv) {
   *scale = s; *inv = i;
 }
 
-struct Source { const float* p; int64_t ld; };
+// The activation scales layer S uses at `bits`: adjusted ones if the adjustment step set them,
+// else the max-calibrated ones.
+inline void act_scales(const LayerState& S, int bits, float* scale, float* inv) {
+  if (S.adj_act[bits]) { *scale = S.adj_sx[bits]; *inv = S.adj_ix[bits]; return; }
+  host_scales(S.act_absmax, bits, scale, inv);
+}
+inline float act_inv(const LayerState& S, int bits) { float s, i; act_scales(S, bits, &s, &i); return i; }
 
 // Row length of the external input: widest slice any layer reads from it (channels for images).
 int64_t ext_ld_of(const Model* M) {
@@ -284,6 +296,17 @@ int64_t ext_ld_of(const Model* M) {
     if (w > ld) ld = w;
   }
   return ld;
+}
+
+// Back to the max-calibrated scales everywhere (after a scale adjustment).
+void reset_adjusted_scales(Model* M) {
+  for (auto& S : M->L) {
+    for (int b = 0; b < 17; ++b) {
+      S.adj_act[b] = false;
+      if (S.wc[b].adjusted) { S.wc[b].adjusted = false; S.wc[b].ready = false; }
+    }
+  }
+  M->reuse_valid = false;
 }
 
 // One forward pass.  calibrate = true: every layer at 16 bit, record max|input| per layer.
@@ -410,7 +433,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       int share = -1;
       for (int j = 0; j < l && share < 0; ++j) {
         LayerState& T = M->L[j];
-        if (same_input(T.d, d) && T.bits == b && T.a_ptr && (b == 16 || T.act_absmax == S.act_absmax) &&
+        if (same_input(T.d, d) && T.bits == b && T.a_ptr && (b == 16 || act_inv(T, b) == act_inv(S, b)) &&
             (dirty[j] || T.a_ptr == T.abuf.p))       // a skipped layer's codes are trusted only in its own buffer
           share = j;
       }
@@ -420,7 +443,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
         rc = S.abuf.ensure(ctx, (size_t)(S.rows * S.ldk) * 2);
         if (rc) return rc;
         float sc = 1.0f, inv = 1.0f;
-        if (b != 16) host_scales(S.act_absmax, b, &sc, &inv);
+        if (b != 16) act_scales(S, b, &sc, &inv);
         if (direct)
           rc = launch_quantize(ctx, tp, S.rows, d.k_in, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
         else
@@ -440,7 +463,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     g.act = S.d.act;
     if (b != 16) {
       float sx, ix;
-      host_scales(S.act_absmax, b, &sx, &ix);
+      act_scales(S, b, &sx, &ix);
       g.scale_x = sx;
       g.scale_w = (const float*)S.wc[b].scale.p;
     }
@@ -453,7 +476,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       const bool fusable = ctx->fuse && !calibrate && reads_rows_directly(C.d) && C.d.src_col0 == 0 && C.d.k_in == S.d.n_out;
       if (!fusable) { all_fused = false; continue; }
       float csc = 1.0f, cinv = 1.0f;
-      if (cb != 16) host_scales(C.act_absmax, cb, &csc, &cinv);
+      if (cb != 16) act_scales(C, cb, &csc, &cinv);
       // an existing slot with the same grid serves this consumer too
       int found = -1;
       for (int s = 0; s < nslots; ++s)
@@ -801,10 +824,14 @@ int qcfg_model_destroy(qcfg_model* model) {
   Model* M = &model->m;
   for (auto& S : M->L) {
     S.w_absmax.release(); S.ybuf.release(); S.abuf.release(); S.prebuf.release();
+    S.ylin.release(); S.yact.release(); S.gout.release(); S.dsw.release(); S.diw.release();
     for (auto& W : S.wc) { W.codes.release(); W.scale.release(); W.inv.release(); }
   }
   M->act_absmax_dev.release();
   M->search_ref.release(); M->search_out.release(); M->search_partial.release();
+  M->noise_codes.release(); M->noise_amax.release();
+  M->adj_gs.release(); M->adj_gt.release(); M->adj_qxt.release(); M->adj_qwt.release();
+  M->adj_dx.release(); M->adj_dw.release(); M->adj_colsum.release(); M->adj_dscal.release();
   delete model;
   return QCFG_OK;
 }
@@ -826,6 +853,7 @@ int qcfg_calibrate_model(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, i
   for (size_t l = 0; l < host.size(); ++l)
     if (!std::isfinite(host[l])) return set_error(c, QCFG_ENONFINITE, "layer %zu: calibrated input maximum is not finite", l);
   for (size_t l = 0; l < host.size(); ++l) M->L[l].act_absmax = host[l];
+  reset_adjusted_scales(M);
   M->calibrated = true;
   M->evaluated = false;
   return QCFG_OK;
@@ -1123,6 +1151,276 @@ int qcfg_noise_sensitivity(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev,
   }
   M->evaluated = true;
   M->last_m = m;
+  return QCFG_OK;
+}
+
+
+// ---- scale adjustment (Section 3.1, second step; learning rate of Section 4) -------------------
+
+namespace {
+
+// One pass of the adjustment: the forward of the model under `bits` with its current scales, layer
+// by layer with the rescaled accumulators (ylin) and the activated outputs (yact) kept, the loss
+// against yref, and (want_grads) the backward pass that leaves the gradients of the weight scales
+// in every layer's dsw / diw and those of the activation scales in M->adj_dscal (two doubles per
+// layer: d/d(scale), d/d(inv_scale)).  Linear layers only.  Synchronises the stream.
+int adjust_pass(qcfg_ctx* h, Model* M, const uint8_t* bits, const float* x_dev, int64_t m, const float* yref, double* loss,
+                bool want_grads, cudaStream_t st) {
+  Ctx* c = &h->c;
+  const int n = (int)M->L.size();
+  const int64_t x_ld = ext_ld_of(M);
+  M->reuse_valid = false;
+  auto input_of = [&](int l, const float** p, int64_t* ld) {
+    const qcfg_layer& d = M->L[l].d;
+    if (d.src < 0) { *p = x_dev + d.src_col0; *ld = x_ld; }
+    else { *p = (const float*)M->L[d.src].yact.p + d.src_col0; *ld = M->L[d.src].d.n_out; }
+  };
+  int rc = QCFG_OK;
+  for (int l = 0; l < n && !rc; ++l) {
+    LayerState& S = M->L[l];
+    const qcfg_layer& d = S.d;
+    if (d.kh > 0 || d.pool_before != QCFG_POOL_NONE)
+      return set_error(c, QCFG_ESHAPE, "scale adjustment covers linear layers only (layer %d is a convolution or pooled)", l);
+    const int b = bits[l];
+    S.rows = m; S.bits = b;
+    rc = ensure_weight_codes(c, S, b, st);
+    if (!rc) rc = S.abuf.ensure(c, (size_t)(m * S.ldk) * 2);
+    if (!rc) rc = S.ylin.ensure(c, (size_t)(m * d.n_out) * 4);
+    if (!rc) rc = S.yact.ensure(c, (size_t)(m * d.n_out) * 4);
+    if (rc) break;
+    const float* xin; int64_t ldx;
+    input_of(l, &xin, &ldx);
+    float sx = 1.0f, ix = 1.0f;
+    if (b != 16) act_scales(S, b, &sx, &ix);
+    rc = launch_quantize(c, xin, m, d.k_in, ldx, nullptr, ix, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
+    if (rc) break;
+    S.a_ptr = S.abuf.p; S.a_ready = true;
+    GemmArgs g{};
+    g.a = S.abuf.p; g.lda = S.ldk; g.b = S.wc[b].codes.p; g.ldb = S.ldk;
+    g.m = m; g.n = d.n_out; g.k = d.k_in; g.is_bf16 = b == 16; g.act = QCFG_ACT_NONE;
+    g.scale_x = sx; g.scale_w = b == 16 ? nullptr : (const float*)S.wc[b].scale.p;
+    g.y = (float*)S.ylin.p; g.ldy = d.n_out;
+    rc = launch_gemm(c, g, st);
+    const float* res = d.residual_from >= 0 ? (const float*)M->L[d.residual_from].yact.p : nullptr;
+    if (!rc) rc = launch_act_apply(c, (const float*)S.ylin.p, res, d.residual_from >= 0 ? M->L[d.residual_from].d.n_out : 0, d.act,
+                                   (float*)S.yact.p, m, d.n_out, st);
+    S.y_ptr = (const float*)S.yact.p; S.y_internal = false;
+  }
+  if (rc) return rc;
+  LayerState& Z = M->L[n - 1];
+  const int64_t out_elems = m * Z.d.n_out;
+  const int blocks = c->sms * 4;
+  rc = M->search_partial.ensure(c, (size_t)blocks * 16);
+  std::vector<double> partial((size_t)blocks * 2);
+  const float* ref = yref ? yref : (const float*)Z.yact.p;
+  if (!rc) rc = launch_sqdiff(c, (const float*)Z.yact.p, ref, out_elems, (double*)M->search_partial.p, blocks, st);
+  if (!rc) rc = check_cuda(c, cudaMemcpyAsync(partial.data(), M->search_partial.p, (size_t)blocks * 16, cudaMemcpyDeviceToHost, st), "adjust: loss copy");
+  if (!rc) rc = qcfg_sync_status(h, st);
+  if (rc) return rc;
+  double d2 = 0.0, r2 = 0.0;
+  for (int i = 0; i < blocks; ++i) { d2 += partial[2 * i]; r2 += partial[2 * i + 1]; }
+  if (loss) *loss = r2 > 0.0 ? d2 / r2 : 0.0;
+  if (!want_grads) return QCFG_OK;
+  if (!(r2 > 0.0)) return set_error(c, QCFG_ESTATE, "scale adjustment: the reference output is all zero");
+
+  // ---- backward
+  int64_t max_n = 0, max_k = 0;
+  for (auto& S : M->L) { max_n = std::max<int64_t>(max_n, S.d.n_out); max_k = std::max<int64_t>(max_k, S.d.k_in); }
+  const int64_t ldm = round_up(m, 8);
+  rc = M->adj_dscal.ensure(c, (size_t)n * 16);
+  if (!rc) rc = M->adj_colsum.ensure(c, (size_t)max_n * 8);
+  if (!rc) rc = M->adj_gs.ensure(c, (size_t)(m * round_up(max_n, 8)) * 2);
+  if (!rc) rc = M->adj_gt.ensure(c, (size_t)(max_n * ldm) * 2);
+  if (!rc) rc = M->adj_qxt.ensure(c, (size_t)(max_k * ldm) * 2);
+  if (!rc) rc = M->adj_qwt.ensure(c, (size_t)(max_k * round_up(max_n, 8)) * 2);
+  if (!rc) rc = M->adj_dx.ensure(c, (size_t)(m * max_k) * 4);
+  if (!rc) rc = M->adj_dw.ensure(c, (size_t)(max_n * max_k) * 4);
+  if (!rc) rc = check_cuda(c, cudaMemsetAsync(M->adj_dscal.p, 0, (size_t)n * 16, st), "adjust: memset");
+  for (int l = 0; l < n && !rc; ++l) {
+    LayerState& S = M->L[l];
+    rc = S.gout.ensure(c, (size_t)(m * S.d.n_out) * 4);
+    if (!rc) rc = S.dsw.ensure(c, (size_t)S.d.n_out * 8);
+    if (!rc) rc = S.diw.ensure(c, (size_t)S.d.n_out * 8);
+    if (!rc) rc = check_cuda(c, cudaMemsetAsync(S.gout.p, 0, (size_t)(m * S.d.n_out) * 4, st), "adjust: memset");
+    if (!rc) rc = check_cuda(c, cudaMemsetAsync(S.dsw.p, 0, (size_t)S.d.n_out * 8, st), "adjust: memset");
+    if (!rc) rc = check_cuda(c, cudaMemsetAsync(S.diw.p, 0, (size_t)S.d.n_out * 8, st), "adjust: memset");
+  }
+  if (!rc) rc = launch_loss_grad(c, (const float*)Z.yact.p, ref, (float)(2.0 / r2), (float*)Z.gout.p, out_elems, st);
+  double* dscal = (double*)M->adj_dscal.p;
+  for (int l = n - 1; l >= 0 && !rc; --l) {
+    LayerState& S = M->L[l];
+    const qcfg_layer& d = S.d;
+    const int b = bits[l];
+    const int64_t nn = d.n_out, kk = d.k_in, ldn = round_up(nn, 8);
+    float* gpre = (float*)S.gout.p;
+    const float* res = d.residual_from >= 0 ? (const float*)M->L[d.residual_from].yact.p : nullptr;
+    const int64_t ldr = d.residual_from >= 0 ? M->L[d.residual_from].d.n_out : 0;
+    rc = launch_act_backward(c, gpre, (const float*)S.ylin.p, res, ldr, d.act, m, nn, st);
+    if (!rc && d.residual_from >= 0)          // the shortcut passes the gradient on unchanged
+      rc = launch_input_backward(c, gpre, nullptr, 0, 1.0f, 1.0f, 0.0f, m, nn, (float*)M->L[d.residual_from].gout.p, ldr, nullptr, st);
+    float sx = 1.0f, ix = 1.0f;
+    if (b != 16) act_scales(S, b, &sx, &ix);
+    const float qm = b == 16 ? 0.0f : qmax_of(b);
+    if (!rc && b != 16) {       // post-rounding scales: d/ds_w[n] = sum_m g*ylin / s_w[n], d/ds_x = sum g*ylin / s_x
+      rc = check_cuda(c, cudaMemsetAsync(M->adj_colsum.p, 0, (size_t)nn * 8, st), "adjust: memset");
+      if (!rc) rc = launch_col_dot(c, gpre, (const float*)S.ylin.p, m, nn, (double*)M->adj_colsum.p, st);
+      if (!rc) rc = launch_gamma_finish(c, (const double*)M->adj_colsum.p, (const float*)S.wc[b].scale.p, sx, nn, (double*)S.dsw.p, dscal + 2 * l, st);
+    }
+    // gradient of the input codes: dxq[m][k] = sum_n (g[m][n] s_w[n]) qw[n][k]   (bf16 tensor-core GEMM)
+    if (!rc) rc = launch_scale_cols_bf16(c, gpre, b == 16 ? nullptr : (const float*)S.wc[b].scale.p, m, nn, M->adj_gs.p, ldn, st);
+    if (!rc) rc = launch_transpose_bf16(c, S.wc[b].codes.p, b == 16 ? 2 : 1, nn, kk, S.ldk, M->adj_qwt.p, ldn, st);
+    if (!rc) {
+      GemmArgs g{};
+      g.a = M->adj_gs.p; g.lda = ldn; g.b = M->adj_qwt.p; g.ldb = ldn;
+      g.m = m; g.n = kk; g.k = nn; g.is_bf16 = 1; g.act = QCFG_ACT_NONE; g.y = (float*)M->adj_dx.p; g.ldy = kk;
+      rc = launch_gemm(c, g, st);
+    }
+    const float* xin; int64_t ldx;
+    input_of(l, &xin, &ldx);
+    float* gprod = d.src >= 0 ? (float*)M->L[d.src].gout.p + d.src_col0 : nullptr;
+    if (!rc) rc = launch_input_backward(c, (const float*)M->adj_dx.p, xin, ldx, sx, ix, qm, m, kk, gprod,
+                                        d.src >= 0 ? M->L[d.src].d.n_out : 0, b == 16 ? nullptr : dscal + 2 * l + 1, st);
+    if (!rc && b != 16) {       // gradient of the weight codes: dwq[n][k] = sum_m g[m][n] qx[m][k], then the pre-rounding scales
+      rc = launch_transpose_bf16(c, gpre, 0, m, nn, nn, M->adj_gt.p, ldm, st);
+      if (!rc) rc = launch_transpose_bf16(c, S.abuf.p, 1, m, kk, S.ldk, M->adj_qxt.p, ldm, st);
+      if (!rc) {
+        GemmArgs g{};
+        g.a = M->adj_gt.p; g.lda = ldm; g.b = M->adj_qxt.p; g.ldb = ldm;
+        g.m = nn; g.n = kk; g.k = m; g.is_bf16 = 1; g.act = QCFG_ACT_NONE; g.y = (float*)M->adj_dw.p; g.ldy = kk;
+        rc = launch_gemm(c, g, st);
+      }
+      if (!rc) rc = launch_weight_alpha(c, (const float*)M->adj_dw.p, d.w_dev, (const float*)S.wc[b].scale.p, (const float*)S.wc[b].inv.p,
+                                        sx, qm, nn, kk, (double*)S.diw.p, st);
+    }
+  }
+  if (!rc) rc = qcfg_sync_status(h, st);
+  return rc;
+}
+
+int adjust_check(Ctx* c, Model* M, const uint8_t* bits, const float* x_dev, int64_t m, const char* who) {
+  if (!bits || !x_dev || m <= 0) return set_error(c, QCFG_EINVAL, "%s: null pointer or m <= 0", who);
+  if (!M->calibrated) return set_error(c, QCFG_ESTATE, "%s: model is not calibrated", who);
+  if ((uintptr_t)x_dev % 4) return set_error(c, QCFG_EALIGN, "%s: x_dev not 4-byte aligned", who);
+  for (size_t l = 0; l < M->L.size(); ++l)
+    if (!bits_ok(bits[l])) return set_error(c, QCFG_EBITS, "%s: layer %zu has bit width %d", who, l, (int)bits[l]);
+  return QCFG_OK;
+}
+
+// reference output: the 16-bit model's last layer, kept in M->search_ref
+int adjust_reference(qcfg_ctx* h, Model* M, const float* x_dev, int64_t m, cudaStream_t st) {
+  Ctx* c = &h->c;
+  const int n = (int)M->L.size();
+  std::vector<uint8_t> b16((size_t)n, 16);
+  int rc = adjust_pass(h, M, b16.data(), x_dev, m, nullptr, nullptr, false, st);
+  const size_t bytes = (size_t)(m * M->L[n - 1].d.n_out) * 4;
+  if (!rc) rc = M->search_ref.ensure(c, bytes);
+  if (!rc) rc = check_cuda(c, cudaMemcpyAsync(M->search_ref.p, M->L[n - 1].yact.p, bytes, cudaMemcpyDeviceToDevice, st), "adjust: reference copy");
+  return rc;
+}
+
+}  // namespace
+
+int qcfg_scale_gradients(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, const float* x_dev, int64_t m,
+                         double* d_scale_x, double* d_inv_scale_x, double* const* d_scale_w, double* const* d_inv_scale_w,
+                         double* loss, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  int rc = adjust_check(c, M, bits, x_dev, m, "scale_gradients");
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int n = (int)M->L.size();
+  rc = adjust_reference(ctx, M, x_dev, m, st);
+  if (!rc) rc = adjust_pass(ctx, M, bits, x_dev, m, (const float*)M->search_ref.p, loss, true, st);
+  if (rc) return rc;
+  std::vector<double> ds((size_t)2 * n);
+  rc = check_cuda(c, cudaMemcpy(ds.data(), M->adj_dscal.p, ds.size() * 8, cudaMemcpyDeviceToHost), "scale_gradients: copy");
+  for (int l = 0; l < n && !rc; ++l) {
+    if (d_scale_x) d_scale_x[l] = bits[l] == 16 ? 0.0 : ds[2 * l];
+    if (d_inv_scale_x) d_inv_scale_x[l] = bits[l] == 16 ? 0.0 : ds[2 * l + 1];
+    const size_t bytes = (size_t)M->L[l].d.n_out * 8;
+    if (d_scale_w && d_scale_w[l]) rc = check_cuda(c, cudaMemcpy(d_scale_w[l], M->L[l].dsw.p, bytes, cudaMemcpyDeviceToHost), "scale_gradients: copy");
+    if (!rc && d_inv_scale_w && d_inv_scale_w[l]) rc = check_cuda(c, cudaMemcpy(d_inv_scale_w[l], M->L[l].diw.p, bytes, cudaMemcpyDeviceToHost), "scale_gradients: copy");
+  }
+  M->evaluated = true; M->last_m = m;
+  return rc;
+}
+
+int qcfg_adjust_scales(qcfg_ctx* ctx, qcfg_model* model, const uint8_t* bits, const float* x_dev, int64_t m, int32_t steps,
+                       double lr, double* losses_host, void* stream) {
+  if (!ctx || !model) return QCFG_EINVAL;
+  Ctx* c = &ctx->c;
+  Model* M = &model->m;
+  int rc = adjust_check(c, M, bits, x_dev, m, "adjust_scales");
+  if (rc) return rc;
+  if (steps < 0 || !(lr >= 0.0) || !std::isfinite(lr)) return set_error(c, QCFG_EINVAL, "adjust_scales: steps and lr must be >= 0");
+  cudaStream_t st = (cudaStream_t)stream;
+  const int n = (int)M->L.size();
+  rc = adjust_reference(ctx, M, x_dev, m, st);
+  if (rc) return rc;
+  // from here on the scales of (layer, bits[layer]) live on their own: start from their current values
+  for (int l = 0; l < n && !rc; ++l) {
+    const int b = bits[l];
+    if (b == 16) continue;
+    LayerState& S = M->L[l];
+    rc = ensure_weight_codes(c, S, b, st);
+    S.wc[b].adjusted = true;
+    if (!S.adj_act[b]) { host_scales(S.act_absmax, b, &S.adj_sx[b], &S.adj_ix[b]); S.adj_act[b] = true; }
+  }
+  std::vector<double> ds((size_t)2 * n);
+  for (int step = 0; step < steps && !rc; ++step) {
+    double loss = 0.0;
+    rc = adjust_pass(ctx, M, bits, x_dev, m, (const float*)M->search_ref.p, &loss, true, st);
+    if (rc) break;
+    if (losses_host) losses_host[step] = loss;
+    rc = check_cuda(c, cudaMemcpy(ds.data(), M->adj_dscal.p, ds.size() * 8, cudaMemcpyDeviceToHost), "adjust_scales: copy");
+    for (int l = 0; l < n && !rc; ++l) {
+      const int b = bits[l];
+      if (b == 16) continue;
+      LayerState& S = M->L[l];
+      S.adj_sx[b] = (float)((double)S.adj_sx[b] - lr * ds[2 * l]);
+      S.adj_ix[b] = (float)((double)S.adj_ix[b] - lr * ds[2 * l + 1]);
+      rc = launch_sgd(c, (float*)S.wc[b].scale.p, (const double*)S.dsw.p, lr, S.d.n_out, st);
+      if (!rc) rc = launch_sgd(c, (float*)S.wc[b].inv.p, (const double*)S.diw.p, lr, S.d.n_out, st);
+      S.wc[b].ready = false;                    // the weight codes follow the new pre-rounding scales
+    }
+  }
+  double loss = 0.0;
+  if (!rc) rc = adjust_pass(ctx, M, bits, x_dev, m, (const float*)M->search_ref.p, &loss, false, st);
+  if (!rc && losses_host) losses_host[steps] = loss;
+  M->evaluated = true; M->last_m = m;
+  M->reuse_valid = false;
+  return rc;
+}
+
+int qcfg_model_scales(qcfg_model* model, int32_t layer, int bits, float* scale_x, float* inv_scale_x, float* scale_w_host,
+                      float* inv_scale_w_host) {
+  if (!model) return QCFG_EINVAL;
+  Model* M = &model->m;
+  Ctx* c = M->ctx;
+  if (layer < 0 || layer >= (int)M->L.size()) return set_error(c, QCFG_EINVAL, "model_scales: bad layer index");
+  if (!bits_int(bits)) return set_error(c, QCFG_EBITS, "model_scales: bits must be 2..8, got %d", bits);
+  if (!M->calibrated) return set_error(c, QCFG_ESTATE, "model_scales: model is not calibrated");
+  LayerState& S = M->L[layer];
+  float sx, ix;
+  act_scales(S, bits, &sx, &ix);
+  if (scale_x) *scale_x = sx;
+  if (inv_scale_x) *inv_scale_x = ix;
+  if (scale_w_host || inv_scale_w_host) {
+    int rc = ensure_weight_codes(c, S, bits, 0);
+    if (!rc) rc = check_cuda(c, cudaStreamSynchronize(0), "model_scales: sync");
+    const size_t bytes = (size_t)S.d.n_out * 4;
+    if (!rc && scale_w_host) rc = check_cuda(c, cudaMemcpy(scale_w_host, S.wc[bits].scale.p, bytes, cudaMemcpyDeviceToHost), "model_scales: copy");
+    if (!rc && inv_scale_w_host) rc = check_cuda(c, cudaMemcpy(inv_scale_w_host, S.wc[bits].inv.p, bytes, cudaMemcpyDeviceToHost), "model_scales: copy");
+    return rc;
+  }
+  return QCFG_OK;
+}
+
+int qcfg_model_reset_scales(qcfg_model* model) {
+  if (!model) return QCFG_EINVAL;
+  cudaDeviceSynchronize();
+  reset_adjusted_scales(&model->m);
   return QCFG_OK;
 }
 

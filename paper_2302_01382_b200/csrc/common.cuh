@@ -67,6 +67,31 @@ int launch_sweep_static(Ctx* ctx, const float* const* w, const int64_t* rows, co
                         int32_t n_tensors, int granularity, int b_lo, int b_hi, double* sse,
                         float* absmax, cudaStream_t st);
 
+// ----- adjust.cu (scale adjustment, Section 3.1 second step) --------------------------
+// y = act(ylin + res) elementwise over [rows x n] (res may be null; ldr its row pitch)
+int launch_act_apply(Ctx* ctx, const float* ylin, const float* res, int64_t ldr, int act, float* y, int64_t rows, int64_t n, cudaStream_t st);
+// g = coef * (y - yref)
+int launch_loss_grad(Ctx* ctx, const float* y, const float* yref, float coef, float* g, int64_t count, cudaStream_t st);
+// g *= act'(ylin + res) in place
+int launch_act_backward(Ctx* ctx, float* g, const float* ylin, const float* res, int64_t ldr, int act, int64_t rows, int64_t n, cudaStream_t st);
+// out[c] += sum_r a[r][c] * b[r][c]   (out must be zeroed by the caller)
+int launch_col_dot(Ctx* ctx, const float* a, const float* b, int64_t rows, int64_t n, double* out, cudaStream_t st);
+// d_sw[c] = colsum[c] / s_w[c];  *d_sx += sum_c colsum[c] / s_x
+int launch_gamma_finish(Ctx* ctx, const double* colsum, const float* s_w, float s_x, int64_t n, double* d_sw, double* d_sx, cudaStream_t st);
+// out[r][c] = bf16(g[r][c] * (col_scale ? col_scale[c] : 1)), columns n..ld-1 zero
+int launch_scale_cols_bf16(Ctx* ctx, const float* g, const float* col_scale, int64_t rows, int64_t n, void* out, int64_t ld, cudaStream_t st);
+// dst[c][r] = bf16(src[r][c]); kind 0 fp32, 1 int8, 2 bf16 source; dst row pitch ld_dst (columns rows..ld_dst-1 zero)
+int launch_transpose_bf16(Ctx* ctx, const void* src, int kind, int64_t rows, int64_t cols, int64_t ld_src, void* dst, int64_t ld_dst, cudaStream_t st);
+// integer layer: mask = |x*inv_x| <= qmax;  *d_ix += s_x * sum dxq*mask*x;  gprod[r][c] += dxq*(s_x*inv_x)*mask
+// 16-bit layer (qmax == 0): gprod += dxq.  gprod may be null (external input).
+int launch_input_backward(Ctx* ctx, const float* dxq, const float* x, int64_t ldx, float s_x, float inv_x, float qmax,
+                          int64_t rows, int64_t k, float* gprod, int64_t ldg, double* d_ix, cudaStream_t st);
+// d_iw[r] = s_x * s_w[r] * sum_c dwq[r][c] * w[r][c] * (|w[r][c]*inv_w[r]| <= qmax)
+int launch_weight_alpha(Ctx* ctx, const float* dwq, const float* w, const float* s_w, const float* inv_w, float s_x, float qmax,
+                        int64_t n, int64_t k, double* d_iw, cudaStream_t st);
+// s[i] = float(double(s[i]) - lr * g[i])
+int launch_sgd(Ctx* ctx, float* s, const double* g, double lr, int64_t n, cudaStream_t st);
+
 // ----- gemm.cu ------------------------------------------------------------------------
 constexpr int kMaxSlots = 3;
 struct CodeSlot {          // one fused re-quantize output of a GEMM epilogue
@@ -114,6 +139,20 @@ __device__ __forceinline__ double warp_sum(double v) {
 // compare above every finite value, so a max over these bits propagates them.
 __device__ __forceinline__ unsigned abs_bits(float x) { return __float_as_uint(x) & 0x7fffffffu; }
 
+// tanh-GELU as y / (1 + exp(-2u)), u = sqrt(2/pi) (y + 0.044715 y^3), which equals
+// 0.5 y (1 + tanh u).  exp(-2u) = 2^(y (c1 + c3 y^2)) with the constants folded; one ex2 and
+// one reciprocal on the special-function unit, five FMA-pipe operations.
+__device__ __forceinline__ float gelu_tanh(float y) {
+  const float c1 = -2.302208198f;            // -2 sqrt(2/pi) log2(e)
+  const float c3 = -0.1029432396f;           // c1 * 0.044715
+  float y2 = y * y;
+  float t = y * fmaf(c3, y2, c1);
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return y * r;
+}
 __host__ __device__ __forceinline__ float qmax_of(int bits) { return (float)((1 << (bits - 1)) - 1); }
 
 }  // namespace qcfg

@@ -253,20 +253,6 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // ---------------------------------------------------------------------------- epilogue math
 
-// tanh-GELU as y / (1 + exp(-2u)), u = sqrt(2/pi) (y + 0.044715 y^3), which equals
-// 0.5 y (1 + tanh u).  exp(-2u) = 2^(y (c1 + c3 y^2)) with the constants folded; one ex2 and
-// one reciprocal on the special-function unit, five FMA-pipe operations.
-__device__ __forceinline__ float gelu_tanh(float y) {
-  const float c1 = -2.302208198f;            // -2 sqrt(2/pi) log2(e)
-  const float c3 = -0.1029432396f;           // c1 * 0.044715
-  float y2 = y * y;
-  float t = y * fmaf(c3, y2, c1);
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
-  float r;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
-  return y * r;
-}
 // int8 code of Eq. 1 in the low byte of the returned word: clamp, then add 1.5*2^23 (a
 // round-half-even at integer granularity); the low mantissa byte is the two's-complement code.
 __device__ __forceinline__ uint32_t code_word(float y, float inv_scale, float qmax) {
