@@ -101,6 +101,13 @@ int qcfg_set_pair_tiles(qcfg_ctx* ctx, int enabled);
  * one kernel.  Results are bit-identical either way.                                        */
 int qcfg_set_grouping(qcfg_ctx* ctx, int enabled);
 
+/* Switches implicit-GEMM convolutions in model evaluations (default on): a convolution that is not a
+ * plain row read (3x3, strided 1x1, ...) and whose input has channels in whole 16-byte chunks takes
+ * the NHWC codes of its input (written by the producer's epilogue where fusion allows) and the GEMM
+ * kernel gathers the patches itself, so no im2col matrix is written or read.  Off: every such
+ * layer's patch matrix is materialised first.  Results are bit-identical either way.        */
+int qcfg_set_implicit_conv(qcfg_ctx* ctx, int enabled);
+
 /* Switches prefix reuse in model evaluations (default off).  On: qcfg_eval_config keeps every
  * layer's buffers from the previous evaluation and, when it is called again with the same x_dev,
  * the same m and no switch changed in between, recomputes only the layers whose bit width changed,

@@ -22,6 +22,7 @@ struct Ctx {
   int fuse = 1;
   int pair = 1;                     // two-CTA GEMM tiles where they apply
   int group = 1;                    // independent GEMMs of equal shape share a launch
+  int implicit = 1;                 // convolutions gather their patches inside the GEMM (no im2col matrix)
   int reuse = 0;                    // evaluations restart at the first layer whose bit width changed
   int64_t epoch = 0;                // bumped by every switch that changes which buffers hold what
   int pair_clusters[2] = {0, 0};
@@ -206,6 +207,7 @@ struct LayerState {
   const float* y_ptr = nullptr;    // where this layer's fp32 output went (nullptr: not materialised)
   bool a_ready = false;
   bool y_internal = false;         // y_ptr is this layer's own buffer (not the caller's)
+  bool implicit = false;           // a_ptr holds the NHWC codes of the input, the GEMM gathers the patches
   int bits = 0;
 };
 
@@ -245,6 +247,9 @@ int64_t layer_rows(const Model* M, int l, int64_t m_ext) {
 bool reads_rows_directly(const qcfg_layer& d) {
   return d.pool_before == QCFG_POOL_NONE && (d.kh == 0 || (d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0));
 }
+// A convolution whose operand the GEMM can gather from the NHWC codes of its input: not a plain
+// row read, and channels in whole 16-byte chunks at either operand width.
+bool implicit_capable(const qcfg_layer& d) { return d.kh > 0 && !reads_rows_directly(d) && d.in_c % 16 == 0 && !(d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0); }
 bool same_input(const qcfg_layer& a, const qcfg_layer& b) {
   return a.src == b.src && a.src_col0 == b.src_col0 && a.k_in == b.k_in && a.kh == b.kh && a.kw == b.kw &&
          a.stride == b.stride && a.pad == b.pad && a.pool_before == b.pool_before && a.in_h == b.in_h &&
@@ -349,6 +354,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     LayerState& S = M->L[l];
     S.rows = layer_rows(M, l, m);
     if (!dirty[l]) continue;                         // buffers and pointers stay as they are
+    S.implicit = ctx->implicit && !calibrate && implicit_capable(S.d);
     const bool codes_kept = reuse && S.bits == bits[l] && S.a_ready && S.a_ptr && S.a_ptr == S.abuf.p &&
                             (S.d.src < 0 || !dirty[S.d.src]);
     if (!codes_kept) { S.a_ready = false; S.a_ptr = nullptr; }
@@ -440,11 +446,13 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       if (share >= 0) {
         S.a_ptr = M->L[share].a_ptr;
       } else {
-        rc = S.abuf.ensure(ctx, (size_t)(S.rows * S.ldk) * 2);
+        rc = S.abuf.ensure(ctx, (size_t)(S.implicit ? srows * d.in_c : S.rows * S.ldk) * 2);
         if (rc) return rc;
         float sc = 1.0f, inv = 1.0f;
         if (b != 16) act_scales(S, b, &sc, &inv);
-        if (direct)
+        if (S.implicit)      // the input tensor's own codes, NHWC; the GEMM gathers the patches
+          rc = launch_quantize(ctx, sp, srows, d.in_c, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, d.in_c, st);
+        else if (direct)
           rc = launch_quantize(ctx, tp, S.rows, d.k_in, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
         else
           rc = launch_im2col_quantize(ctx, sp, m, d.in_h, d.in_w, d.in_c, d.kh, d.kw, d.stride, d.pad, inv, b, S.abuf.p, S.ldk, st);
@@ -461,6 +469,11 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     g.m = S.rows; g.n = S.d.n_out; g.k = S.d.k_in;
     g.is_bf16 = b == 16;
     g.act = S.d.act;
+    if (S.implicit) {
+      g.lda = d.in_c;
+      g.conv_kh = d.kh; g.conv_kw = d.kw; g.conv_stride = d.stride; g.conv_pad = d.pad;
+      g.conv_h = d.in_h; g.conv_w = d.in_w; g.conv_c = d.in_c;
+    }
     if (b != 16) {
       float sx, ix;
       act_scales(S, b, &sx, &ix);
@@ -473,21 +486,26 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     for (int c : S.consumers) {
       LayerState& C = M->L[c];
       const int cb = calibrate ? 16 : bits[c];
-      const bool fusable = ctx->fuse && !calibrate && reads_rows_directly(C.d) && C.d.src_col0 == 0 && C.d.k_in == S.d.n_out;
+      // a consumer whose operand is this whole output: a plain row read, or a convolution the GEMM gathers for
+      const bool c_implicit = ctx->implicit && !calibrate && implicit_capable(C.d) && C.d.pool_before == QCFG_POOL_NONE;
+      const bool fusable = ctx->fuse && !calibrate && C.d.src_col0 == 0 &&
+                           ((reads_rows_directly(C.d) && C.d.k_in == S.d.n_out) || (c_implicit && C.d.in_c == S.d.n_out));
       if (!fusable) { all_fused = false; continue; }
+      const int64_t c_ld = c_implicit ? C.d.in_c : C.ldk;
       float csc = 1.0f, cinv = 1.0f;
       if (cb != 16) act_scales(C, cb, &csc, &cinv);
       // an existing slot with the same grid serves this consumer too
       int found = -1;
       for (int s = 0; s < nslots; ++s)
-        if ((cb == 16 && g.slots[s].kind == 2) || (cb != 16 && g.slots[s].kind == 1 && g.slots[s].inv_scale == cinv && g.slots[s].qmax == qmax_of(cb)))
+        if (g.slots[s].ld == c_ld &&
+            ((cb == 16 && g.slots[s].kind == 2) || (cb != 16 && g.slots[s].kind == 1 && g.slots[s].inv_scale == cinv && g.slots[s].qmax == qmax_of(cb))))
           found = s;
       if (found < 0) {
         if (nslots == kMaxSlots) { all_fused = false; continue; }
-        rc = C.abuf.ensure(ctx, (size_t)(S.rows * C.ldk) * 2);
+        rc = C.abuf.ensure(ctx, (size_t)(S.rows * c_ld) * 2);
         if (rc) return rc;
         g.slots[nslots].ptr = C.abuf.p;
-        g.slots[nslots].ld = C.ldk;
+        g.slots[nslots].ld = c_ld;
         g.slots[nslots].inv_scale = cinv;
         g.slots[nslots].qmax = cb == 16 ? 0.0f : qmax_of(cb);
         g.slots[nslots].kind = cb == 16 ? 2 : 1;
@@ -496,6 +514,7 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       C.a_ptr = g.slots[found].ptr;
       C.a_ready = true;
       C.bits = cb;
+      C.implicit = c_implicit;
     }
     float* y_out = (y_dev && y_dev[l]) ? y_dev[l] : nullptr;
     const bool need_y = y_out || !all_fused || S.feeds_residual;
@@ -647,6 +666,12 @@ int qcfg_set_grouping(qcfg_ctx* ctx, int enabled) {
 int qcfg_set_fusion(qcfg_ctx* ctx, int enabled) {
   if (!ctx) return QCFG_EINVAL;
   ctx->c.fuse = enabled ? 1 : 0;
+  ctx->c.epoch++;
+  return QCFG_OK;
+}
+int qcfg_set_implicit_conv(qcfg_ctx* ctx, int enabled) {
+  if (!ctx) return QCFG_EINVAL;
+  ctx->c.implicit = enabled ? 1 : 0;
   ctx->c.epoch++;
   return QCFG_OK;
 }
@@ -1434,7 +1459,12 @@ int qcfg_debug_dump(qcfg_ctx* ctx, qcfg_model* model, int32_t layer, int8_t* qx_
   LayerState& S = M->L[layer];
   if (!bits_int(S.bits)) return set_error(c, QCFG_EBITS, "debug_dump: layer %d ran at %d bit", layer, S.bits);
   cudaStream_t st = (cudaStream_t)stream;
-  if (qx_dev) {
+  if (qx_dev && S.implicit) {     // the patches were never materialised: gather them from the input's codes now
+    const qcfg_layer& d = S.d;
+    const int64_t opix = (int64_t)((d.in_h + 2 * d.pad - d.kh) / d.stride + 1) * ((d.in_w + 2 * d.pad - d.kw) / d.stride + 1);
+    int rc = launch_im2col_codes(c, (const int8_t*)S.a_ptr, S.rows / opix, d.in_h, d.in_w, d.in_c, d.kh, d.kw, d.stride, d.pad, qx_dev, d.k_in, st);
+    if (rc) return rc;
+  } else if (qx_dev) {
     cudaError_t e = cudaMemcpy2DAsync(qx_dev, (size_t)S.d.k_in, S.a_ptr, (size_t)S.ldk, (size_t)S.d.k_in, (size_t)S.rows, cudaMemcpyDeviceToDevice, st);
     if (e != cudaSuccess) return check_cuda(c, e, "debug_dump qx copy");
   }
@@ -1446,6 +1476,12 @@ int qcfg_debug_dump(qcfg_ctx* ctx, qcfg_model* model, int32_t layer, int8_t* qx_
     GemmArgs g{};
     g.a = S.a_ptr; g.lda = S.ldk; g.b = S.wc[S.bits].codes.p; g.ldb = S.ldk;
     g.m = S.rows; g.n = S.d.n_out; g.k = S.d.k_in; g.acc = acc_dev;
+    if (S.implicit) {
+      const qcfg_layer& d = S.d;
+      g.lda = d.in_c;
+      g.conv_kh = d.kh; g.conv_kw = d.kw; g.conv_stride = d.stride; g.conv_pad = d.pad;
+      g.conv_h = d.in_h; g.conv_w = d.in_w; g.conv_c = d.in_c;
+    }
     g.scale_x = 1.0f; g.scale_w = (const float*)S.wc[S.bits].scale.p;
     return launch_gemm(c, g, st);
   }

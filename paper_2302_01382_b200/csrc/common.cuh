@@ -57,6 +57,10 @@ int launch_avgpool(Ctx* ctx, const float* src, int64_t B, int HW, int C, float* 
 int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, int C, int kh, int kw, int stride,
                            int pad, float inv_scale, int bits, void* q, int64_t ldq, cudaStream_t st);
 
+// patches of int8 codes in (kh, kw, cin) order: dst [B*OH*OW x ldd] from NHWC codes [B*H*W x C] (C % 16 == 0)
+int launch_im2col_codes(Ctx* ctx, const int8_t* src, int64_t B, int H, int W, int C, int kh, int kw, int stride, int pad,
+                        int8_t* dst, int64_t ldd, cudaStream_t st);
+
 // ----- sweep.cu -----------------------------------------------------------------------
 int sweep_init(Ctx* ctx);   // per-device kernel attributes
 int launch_sweep(Ctx* ctx, const float* const* w, const int64_t* rows, const int64_t* cols,
@@ -113,6 +117,9 @@ struct GemmArgs {
   const float* residual; int64_t ldr;  // optional fp32 addend (before act)
   int32_t* acc;                 // optional raw accumulators (int8 only) [m x n]
   CodeSlot slots[kMaxSlots];
+  // implicit-GEMM convolution (conv_kh > 0): `a` is the NHWC code tensor [batch*H*W x C] of the layer's
+  // input (lda = C), m = batch*OH*OW, k = kh*kw*C; the kernel gathers the patches itself
+  int conv_kh = 0, conv_kw = 0, conv_stride = 0, conv_pad = 0, conv_h = 0, conv_w = 0, conv_c = 0;
 };
 int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st);
 // up to three GEMMs of equal m, k, operand type and tile width in one launch

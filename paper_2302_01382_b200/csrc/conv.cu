@@ -212,4 +212,40 @@ int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, 
   return check_cuda(ctx, cudaGetLastError(), "im2col launch");
 }
 
+
+// Patches of an int8 NHWC code tensor (parity taps of convolutions whose GEMM gathers its operand
+// itself): one thread per 16 codes of an output row.
+__global__ void __launch_bounds__(256) im2col_codes_kernel(const int8_t* __restrict__ src, int64_t rows, int H, int W, int C, int kh,
+                                                           int kw, int stride, int pad, int OH, int OW, int8_t* __restrict__ dst,
+                                                           int64_t ldd) {
+  const int cpr = kh * kw * C / 16;                 // 16-code chunks per output row
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * cpr) return;
+  const int64_t row = idx / cpr;
+  const int k0 = (int)(idx - row * cpr) * 16;
+  const int tap = k0 / C, c = k0 - tap * C, dy = tap / kw, dx = tap - dy * kw;
+  const int64_t b = row / ((int64_t)OH * OW);
+  const int pix = (int)(row - b * OH * OW), oh = pix / OW, ow = pix - oh * OW;
+  const int ih = oh * stride - pad + dy, iw = ow * stride - pad + dx;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (ih >= 0 && ih < H && iw >= 0 && iw < W)
+    v = *reinterpret_cast<const uint4*>(src + ((b * H + ih) * W + iw) * C + c);
+  int8_t* o = dst + row * ldd + k0;
+  if ((reinterpret_cast<uintptr_t>(o) & 15) == 0) *reinterpret_cast<uint4*>(o) = v;
+  else {
+    const int8_t* pv = reinterpret_cast<const int8_t*>(&v);
+    for (int j = 0; j < 16; ++j) o[j] = pv[j];
+  }
+}
+
+int launch_im2col_codes(Ctx* ctx, const int8_t* src, int64_t B, int H, int W, int C, int kh, int kw, int stride, int pad,
+                        int8_t* dst, int64_t ldd, cudaStream_t st) {
+  const int OH = (H + 2 * pad - kh) / stride + 1, OW = (W + 2 * pad - kw) / stride + 1;
+  const int64_t rows = B * OH * OW, total = rows * (kh * kw * C / 16);
+  if (total == 0) return QCFG_OK;
+  im2col_codes_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(src, rows, H, W, C, kh, kw, stride, pad, OH, OW, dst, ldd);
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "code patch launch");
+}
+
 }  // namespace qcfg

@@ -29,6 +29,9 @@ constexpr int kStageKBytes = 128;     // bytes of K per stage row = one 128B swi
 constexpr int kUmmaKBytes = 32;       // bytes of K per tcgen05.mma
 constexpr int kEpiWarps = 16;
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+constexpr int kGatherWarps = 2;       // convolution launches only: build the A tile from the NHWC source
+constexpr int kGemmThreadsConv = kGemmThreads + 32 * kGatherWarps;
+constexpr int kGatherDepth = 2;       // k-blocks a gather warp keeps in flight
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;         // columns per accumulator buffer
 constexpr int kMaxStages = 8;
@@ -69,6 +72,14 @@ struct GroupDesc {
   const float* residual; int64_t ldr;
   OutDesc outs[kNumOuts];     // [0] raw accumulators, [1] fp32 output, [2..] consumer codes
 };
+// Implicit-GEMM convolution: the A operand is not a matrix in memory but the NHWC code tensor of the
+// layer's input; row (b, oh, ow) of the k-block (tap, channel chunk) is gathered from pixel
+// (b, oh*stride - pad + dy, ow*stride - pad + dx), zero outside the image.
+struct ConvDesc {
+  int32_t on, H, W, C, kh, kw, stride, pad, OH, OW, esz, K;
+  int64_t img_bytes;          // bytes of one image (H * W * C * esz)
+  const uint8_t* src;
+};
 struct GemmParams {
   int32_t m, k_blocks, bn, tiles_m, tiles_n, stages, is_bf16;   // tiles_n: column tiles of all groups together
   int32_t epi_bytes;          // staging bytes per epilogue warp (2048 or 4096)
@@ -76,6 +87,7 @@ struct GemmParams {
   GroupDesc grp[kMaxGroups];  // unused groups have tn_begin = INT32_MAX
   unsigned* err;
   unsigned long long* stamp;  // optional [2]: earliest start / latest end of the launch's CTAs (%globaltimer, ns)
+  ConvDesc conv;              // conv.on: A comes from the gather warps (single-group launches only)
 };
 
 // ---------------------------------------------------------------------------- PTX wrappers
@@ -530,7 +542,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
 // ---------------------------------------------------------------------------- the kernel
 
 template <bool BF16, bool PAIR, bool GROUPED>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreadsConv, 1)
 gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the 128B swizzle atoms
@@ -590,16 +602,19 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   };
   set_tile_coords();
   const bool elected = elect_one();    // the lane of a converged warp that issues TMA / MMA instructions
+  const bool conv_on = p.conv.on != 0;
+  // bytes the TMA loads of one CTA put into a stage (the A tile is gathered in convolution launches)
+  const uint32_t tma_bytes = conv_on ? (uint32_t)b_rows * kStageKBytes : stage_bytes;
   auto issue_load = [&]() {   // whole warp 0; the stage's empty barrier must already have been passed
     if (elected) {
     if (PAIR) {
       // the first CTA's barrier collects the bytes of both CTAs' loads
-      if (rank == 0) mbar_expect_tx(ld_bar, 2 * stage_bytes);
-      tma_load_2d_pair(ld_dst, ld_map_a, ld_bar, ld_x, ld_ya);
+      if (rank == 0) mbar_expect_tx(ld_bar, 2 * tma_bytes);
+      if (!conv_on) tma_load_2d_pair(ld_dst, ld_map_a, ld_bar, ld_x, ld_ya);
       tma_load_2d_pair(ld_dst + BM * kStageKBytes, ld_map_b, ld_bar, ld_x, ld_yb);
     } else {
-      mbar_expect_tx(ld_bar, stage_bytes);
-      tma_load_2d(ld_dst, ld_map_a, ld_bar, ld_x, ld_ya);
+      mbar_expect_tx(ld_bar, tma_bytes);
+      if (!conv_on) tma_load_2d(ld_dst, ld_map_a, ld_bar, ld_x, ld_ya);
       tma_load_2d(ld_dst + BM * kStageKBytes, ld_map_b, ld_bar, ld_x, ld_yb);
     }
     }
@@ -616,7 +631,8 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.g[0].a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.g[0].b) : "memory");
-    for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    const uint32_t full_count = 1 + (p.conv.on ? kGatherWarps * (PAIR ? 2 : 1) : 0);   // the TMA thread, plus one arrival per gather warp
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -710,6 +726,74 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
         if (ok && elected) { if (PAIR) tc_commit_pair(tfull0 + 8 * a); else tc_commit(tfull0 + 8 * a); }   // accumulator complete
       }
     }
+  } else if (warp >= 2 + kEpiWarps) {
+    // ------------------------------------------------------------------ gather warps (convolutions)
+    // Each lane owns two rows of the CTA's 128-row A tile.  Per k-block it copies the rows' eight
+    // 16-byte chunks from the NHWC source (cp.async with zero fill outside the image, beyond the
+    // reduction length and past the last row) to where a 128B-swizzled TMA box would have put them.
+    // kGatherDepth k-blocks stay in flight; when the oldest has landed the lane makes its writes
+    // visible to the tensor core (fence.proxy.async) and one lane per warp arrives on the stage's
+    // full barrier (the pair's first CTA's).
+    const ConvDesc& cv = p.conv;
+    const int gw = warp - (2 + kEpiWarps);
+    const int epc = 16 / cv.esz;                       // elements per 16-byte chunk
+    const int opix = cv.OH * cv.OW;
+    int s = 0, as = 0, inflight = 0;
+    uint32_t ph = 0;
+    int tm = tm0, tn = tn0;
+    bool ok = true;
+    auto landed = [&]() {                              // the oldest group in flight has landed
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) { if (PAIR) mbar_arrive_leader(full0 + 8 * as); else mbar_arrive(full0 + 8 * as); }
+      if (++as == p.stages) as = 0;
+      --inflight;
+    };
+    for (int tile = tile0; tile < num_tiles && ok; tile += tile_step) {
+      int ih0[2], iw0[2];
+      const uint8_t* img[2];
+      bool rv[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int64_t pm = (int64_t)tm * rows_per_tile + rank * BM + gw * 64 + i * 32 + lane;
+        rv[i] = pm < p.m;
+        const int q = rv[i] ? (int)pm : 0;
+        const int b = q / opix, pix = q - b * opix;
+        const int oh = pix / cv.OW, ow = pix - oh * cv.OW;
+        ih0[i] = oh * cv.stride - cv.pad;
+        iw0[i] = ow * cv.stride - cv.pad;
+        img[i] = cv.src + (int64_t)b * cv.img_bytes;
+      }
+      int dy = 0, dx = 0, c = 0, ke = 0;
+      for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+        if (!mbar_wait_warp(empty0 + 8 * s, ph ^ 1, abort_flag, p.err)) { ok = false; break; }
+        const uint32_t a_dst = stage0 + (uint32_t)s * stage_bytes + (uint32_t)(gw * 64 + lane) * 128;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const bool kin = ke < cv.K;
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const int ih = ih0[i] + dy, iw = iw0[i] + dx;
+            const bool valid = rv[i] && kin && (unsigned)ih < (unsigned)cv.H && (unsigned)iw < (unsigned)cv.W;
+            const uint8_t* src = valid ? img[i] + ((int64_t)(ih * cv.W + iw) * cv.C + c) * cv.esz : cv.src;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                         ::"r"(a_dst + i * 32 * 128 + ((j ^ (lane & 7)) << 4)), "l"(src), "r"(valid ? 16 : 0) : "memory");
+          }
+          ke += epc; c += epc;
+          if (c >= cv.C) { c = 0; if (++dx == cv.kw) { dx = 0; ++dy; } }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (++s == p.stages) { s = 0; ph ^= 1; }
+        if (++inflight > kGatherDepth) {
+          asm volatile("cp.async.wait_group %0;" ::"n"(kGatherDepth) : "memory");
+          landed();
+        }
+      }
+      tm += step_tm; tn += step_tn;
+      if (tm >= p.tiles_m) { tm -= p.tiles_m; ++tn; }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    while (inflight > 0) landed();
   } else {
     // ------------------------------------------------------------------ epilogue
     const int ew = warp - 2;
@@ -924,6 +1008,7 @@ int gemm_init(Ctx* ctx) {
 static int tile_n_of(int64_t n) { return n <= 32 ? 32 : n <= 64 ? 64 : n <= 128 ? 128 : 256; }
 
 bool gemm_groupable(const GemmArgs& a, const GemmArgs& b) {
+  if (a.conv_kh > 0 || b.conv_kh > 0) return false;
   return a.m == b.m && a.k == b.k && a.is_bf16 == b.is_bf16 && tile_n_of(a.n) == tile_n_of(b.n);
 }
 
@@ -937,7 +1022,12 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
     if (g.m <= 0 || g.n <= 0 || g.k <= 0) return set_error(ctx, QCFG_ESHAPE, "gemm: m, n, k must be positive");
     if (((uintptr_t)g.a & 15) || ((uintptr_t)g.b & 15) || (g.lda * esz) % 16 || (g.ldb * esz) % 16)
       return set_error(ctx, QCFG_EALIGN, "gemm: operands need 16-byte aligned pointers and row strides");
-    if (g.lda < g.k || g.ldb < g.k) return set_error(ctx, QCFG_ESHAPE, "gemm: leading dimension below k");
+    if (g.conv_kh > 0) {
+      if (count > 1) return set_error(ctx, QCFG_EINVAL, "gemm: convolutions are launched alone");
+      if ((g.conv_c * esz) % 16 || g.lda != g.conv_c || g.k != (int64_t)g.conv_kh * g.conv_kw * g.conv_c || g.conv_stride < 1)
+        return set_error(ctx, QCFG_ESHAPE, "gemm: convolution needs channels in whole 16-byte chunks and k = kh*kw*c");
+      if (g.ldb < g.k) return set_error(ctx, QCFG_ESHAPE, "gemm: leading dimension below k");
+    } else if (g.lda < g.k || g.ldb < g.k) return set_error(ctx, QCFG_ESHAPE, "gemm: leading dimension below k");
     if (g.m > 0x7fffffff || g.n > 0x7fffffff) return set_error(ctx, QCFG_ESHAPE, "gemm: dimension too large");
     if (i && !gemm_groupable(g0, g)) return set_error(ctx, QCFG_EINVAL, "gemm: grouped launches need equal m, k, type and tile width");
   }
@@ -994,15 +1084,28 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       if (!G.outs[1].kind && G.outs[2].kind == 1 && make_fast_map(&maps.g[i].fast, G.outs[2], g.m, g.n)) G.mode = EPI_CODES1;
       else if (G.outs[1].kind && !G.outs[2].kind && make_fast_map(&maps.g[i].fast, G.outs[1], g.m, g.n)) { G.mode = EPI_Y; wide = true; }
     }
-    int rc = make_map(ctx, &maps.g[i].a, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
+    int rc = g.conv_kh > 0 ? QCFG_OK : make_map(ctx, &maps.g[i].a, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
     if (rc == QCFG_OK) rc = make_map(ctx, &maps.g[i].b, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
     if (rc != QCFG_OK) return rc;
     ops += 2.0 * (double)g.m * (double)g.n * (double)g.k;
   }
   p.tiles_n = tn_total;
+  const bool conv = g0.conv_kh > 0;
+  if (conv) {
+    ConvDesc& cv = p.conv;
+    cv.on = 1; cv.H = g0.conv_h; cv.W = g0.conv_w; cv.C = g0.conv_c; cv.kh = g0.conv_kh; cv.kw = g0.conv_kw;
+    cv.stride = g0.conv_stride; cv.pad = g0.conv_pad; cv.esz = esz; cv.K = (int32_t)g0.k;
+    cv.OH = (cv.H + 2 * cv.pad - cv.kh) / cv.stride + 1;
+    cv.OW = (cv.W + 2 * cv.pad - cv.kw) / cv.stride + 1;
+    cv.img_bytes = (int64_t)cv.H * cv.W * cv.C * esz;
+    cv.src = reinterpret_cast<const uint8_t*>(g0.a);
+    if (cv.OH < 1 || cv.OW < 1 || g0.m % ((int64_t)cv.OH * cv.OW))
+      return set_error(ctx, QCFG_ESHAPE, "gemm: convolution rows are not a whole number of images");
+  }
   p.epi_bytes = wide ? 4096 : 2048;
   int stages = (kSmemMax - kSmemHeader - kCsBytes - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (stages <= kGatherDepth) return set_error(ctx, QCFG_ESHAPE, "gemm: too few pipeline stages");
   p.stages = stages;
 
   const int num_tiles = p.tiles_m * p.tiles_n;
@@ -1034,7 +1137,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
   // touching global memory.
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kGemmThreads);
+  cfg.blockDim = dim3(conv ? kGemmThreadsConv : kGemmThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];

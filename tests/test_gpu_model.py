@@ -254,3 +254,30 @@ def test_resnet_small_teacher_forced(ctx, fuse):
         model.close()
     finally:
         ctx.set_fusion(True)
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+def test_implicit_and_materialised_convolutions_agree_bitwise(ctx, fuse):
+    """The GEMM that gathers its patches from the input's NHWC codes gives, layer by layer, the same
+    bits as the GEMM on a materialised patch matrix: 3x3 with stride 1 and 2, strided 1x1, channel
+    counts of one to several 16-byte chunks, int8 and 16-bit layers, ragged last row tiles."""
+    for width, batch, hw in ((16, 3, 64), (48, 2, 40)):
+        w = wl.resnet50(seed=5, batch=batch, in_hw=hw, width=width, n_classes=10, blocks=(2, 1, 1, 1))
+        model, x = build(ctx, w)
+        model.calibrate_model(x, w.m)
+        n = len(w.layers)
+        with16 = np.array(w.bits).copy()
+        with16[3::4] = 16
+        for bits in (w.bits, [8] * n, with16):
+            outs = {}
+            for implicit in (True, False):
+                ctx.set_implicit_conv(implicit)
+                ctx.set_fusion(fuse)
+                ys = run_eval(ctx, model, w, x, bits)
+                outs[implicit] = [host(y) for y in ys]
+            for l in range(n):
+                np.testing.assert_array_equal(outs[True][l].view(np.uint32), outs[False][l].view(np.uint32),
+                                              err_msg=f"width {width} layer {l} ({w.layers[l].name})")
+        ctx.set_implicit_conv(True)
+        ctx.set_fusion(True)
+        model.close()
