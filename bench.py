@@ -246,6 +246,13 @@ def timed_evals(torch, ctx, model, configs, x, m, ys, reps: int):
     l0 = ctx.launch_count()
     ctx.profile_enable(2)
     ctx.profile_read(0); ctx.profile_read(1)
+    t_host = time.perf_counter()
+    for bits in configs[:2]:                          # host cost: two calls into an empty launch queue
+        model.eval_config(bits, x, m, ys)
+    t_host = (time.perf_counter() - t_host) / len(configs[:2])
+    torch.cuda.synchronize()
+    ctx.profile_read(0); ctx.profile_read(1)
+    l0 = ctx.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(reps):
@@ -259,7 +266,7 @@ def timed_evals(torch, ctx, model, configs, x, m, ys, reps: int):
     n = reps * len(configs)
     ms = e0.elapsed_time(e1) / n
     k_ms = i_ms + b_ms
-    return {"evals_per_s": 1e3 / ms, "ms_per_eval": ms, "evals_timed": n,
+    return {"evals_per_s": 1e3 / ms, "ms_per_eval": ms, "evals_timed": n, "host_enqueue_ms_per_eval": 1e3 * t_host,
             "gemm_tops": (i_ops + b_ops) / (k_ms * 1e-3) / 1e12 if k_ms else None,
             "gemm_int8_tops": i_ops / (i_ms * 1e-3) / 1e12 if i_ms else None,
             "gemm_bf16_tflops": b_ops / (b_ms * 1e-3) / 1e12 if b_ms else None,
@@ -361,6 +368,15 @@ def run_gpu(args):
     g_ms, g_n, g_ops = ctx.profile_read(0)
     b_ms, b_n, b_ops = ctx.profile_read(1)
     ctx.profile_enable(0)
+    # host cost of one evaluation: a few calls into an empty launch queue (a full queue would make
+    # the call wait for the device and show the device's time instead)
+    torch.cuda.synchronize()
+    cfg8 = [8] * len(w.layers)
+    t0 = time.perf_counter()
+    for _ in range(4):
+        job.model.eval_config(cfg8, job.x, w.m, job.ys)
+    host_enqueue_ms = 1e3 * (time.perf_counter() - t0) / 4
+    torch.cuda.synchronize()
 
     # ---------------- one more step with CUDA events around every launch: shares of the kernel
     # classes (the events serialise launches that otherwise overlap, so this step is slower)
@@ -500,6 +516,8 @@ def run_gpu(args):
                        "l2": "inputs larger than L2 (340 MB weights, 38 MB activations per layer)",
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": clocks, "gpu_launches": int(launches),
+            "host": {"enqueue_ms_per_eval": host_enqueue_ms, "device_ms_per_eval": ms_total / args.steps / N_EVALS,
+                     "note": "host time of one qcfg_eval_config call (planning, tensor maps, 48 launches) against the device time it hides behind"},
             "e2e": e2e, "launches_before_timed": int(launches0),
             "roofline": {"kernel": "gemm_kernel<int8>", "bound": "tensor", "achieved": achieved, "peak": sustained2,
                          "unit": "TOP/s", "frac": achieved / sustained2,
