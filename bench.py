@@ -37,7 +37,7 @@ TOKENS = 32 * 384
 WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
 # DRAM bytes (read + write) per int8 GEMM launch from the ncu capture summarised in
 # profiles/gemm_int8_bert_base_block.md; set to None whenever the GEMM kernel changes.
-GEMM_TRAFFIC_BYTES = 27.0e6
+GEMM_TRAFFIC_BYTES = 27.3e6
 DATASHEET_INT8_TOPS = 4500.0      # B200 dense int8, vendor datasheet (an outside figure)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
