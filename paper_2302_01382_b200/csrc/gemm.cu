@@ -17,6 +17,8 @@
 #include <cuda.h>
 
 #include <cstring>
+#include <mutex>
+#include <unordered_map>
 
 #include "common.cuh"
 
@@ -910,17 +912,55 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
+// A two-dimensional tiled tensor map.  Encoding one costs a driver call of a microsecond or two and
+// an evaluation needs a couple of hundred, always the same ones (a map depends only on address,
+// shape, pitch, box, type and swizzle), so encoded maps are kept in a process-wide table.
+struct MapKey {
+  const void* ptr; uint64_t d0, d1, pitch; uint32_t b0, b1, dt, swz, promo;
+  bool operator==(const MapKey& o) const {
+    return ptr == o.ptr && d0 == o.d0 && d1 == o.d1 && pitch == o.pitch && b0 == o.b0 && b1 == o.b1 && dt == o.dt &&
+           swz == o.swz && promo == o.promo;
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    uint64_t h = (uint64_t)(uintptr_t)k.ptr * 0x9E3779B97F4A7C15ull;
+    auto mix = [&](uint64_t v) { h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2); };
+    mix(k.d0); mix(k.d1); mix(k.pitch); mix(((uint64_t)k.b0 << 32) | k.b1); mix(((uint64_t)k.dt << 40) | ((uint64_t)k.swz << 20) | k.promo);
+    return (size_t)h;
+  }
+};
+std::mutex g_map_mutex;
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_map_cache;
+constexpr size_t kMapCacheMax = 16384;
+
+bool encode_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* ptr, uint64_t d0, uint64_t d1, uint64_t pitch_bytes,
+               uint32_t b0, uint32_t b1, CUtensorMapSwizzle swz, CUtensorMapL2promotion promo) {
+  const MapKey key{ptr, d0, d1, pitch_bytes, b0, b1, (uint32_t)dt, (uint32_t)swz, (uint32_t)promo};
+  {
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    auto it = g_map_cache.find(key);
+    if (it != g_map_cache.end()) { *map = it->second; return true; }
+  }
+  cuuint64_t dims[2] = {d0, d1};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {b0, b1};
+  cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode(map, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, promo,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  std::lock_guard<std::mutex> lock(g_map_mutex);
+  if (g_map_cache.size() >= kMapCacheMax) g_map_cache.clear();
+  g_map_cache.emplace(key, *map);
+  return true;
+}
+
 int make_map(Ctx* ctx, CUtensorMap* map, const void* ptr, int is_bf16, int64_t k, int64_t rows, int64_t ld, int box_rows) {
   const int esz = is_bf16 ? 2 : 1;
-  cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)(ld * esz)};
-  cuuint32_t box[2] = {(cuuint32_t)(kStageKBytes / esz), (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(map, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
-                        const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return set_error(ctx, QCFG_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  if (!encode_2d(map, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, ptr, (uint64_t)k, (uint64_t)rows,
+                 (uint64_t)(ld * esz), (uint32_t)(kStageKBytes / esz), (uint32_t)box_rows, CU_TENSOR_MAP_SWIZZLE_128B,
+                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+    return set_error(ctx, QCFG_ECUDA, "cuTensorMapEncodeTiled failed");
   return QCFG_OK;
 }
 
@@ -935,14 +975,8 @@ bool make_out_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
     default: esz = 4; dt = CU_TENSOR_MAP_DATA_TYPE_INT32; break;
   }
   if (((uintptr_t)o.ptr & 15) || ((o.ld * esz) & 15)) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)m};
-  cuuint64_t strides[1] = {(cuuint64_t)(o.ld * esz)};
-  cuuint32_t box[2] = {esz == 4 ? 16u : 32u, 32};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(map, dt, 2, o.ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        esz == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return encode_2d(map, dt, o.ptr, (uint64_t)n, (uint64_t)m, (uint64_t)(o.ld * esz), esz == 4 ? 16u : 32u, 32u,
+                   esz == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
 // Tensor map of the output a fast epilogue body writes: 32-row boxes of 64 int8 columns (64B
@@ -951,15 +985,9 @@ bool make_fast_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
   const bool codes = o.kind == 1;
   const int esz = codes ? 1 : 4;
   if (((uintptr_t)o.ptr & 15) || ((o.ld * esz) & 15)) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)n, (cuuint64_t)m};
-  cuuint64_t strides[1] = {(cuuint64_t)(o.ld * esz)};
-  cuuint32_t box[2] = {codes ? 64u : 32u, 32};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(map, codes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, o.ptr, dims,
-                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        codes ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return encode_2d(map, codes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, o.ptr, (uint64_t)n, (uint64_t)m,
+                   (uint64_t)(o.ld * esz), codes ? 64u : 32u, 32u, codes ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
 // Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on, with
