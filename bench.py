@@ -304,6 +304,10 @@ def other_workloads(torch, q, ctx, peaks):
         res.update(timed_evals(torch, ctx, model, cfgs, x, w.m, ys, reps))
         res["bits"] = sorted(set(int(b) for c in cfgs for b in c))
         res["layers"] = len(w.layers)
+        act_mb = 4.0 * max(wl.layer_rows(w.layers, l, w.m) * lay.n_out for l, lay in enumerate(w.layers)) / 1e6
+        wt_mb = 4.0 * sum(a.size for a in w.weights) / 1e6
+        res["l2"] = ("inputs larger than L2" if wt_mb + act_mb > 126.0 else
+                     "working set fits the 126 MB L2: an L2-resident figure (no flush between evaluations)")
         out[name] = res
         model.close()
         del weights, x, ys
