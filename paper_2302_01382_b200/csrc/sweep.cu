@@ -109,6 +109,11 @@ sweep_rows_kernel(const SweepSeg* __restrict__ segs, const SweepBlock* __restric
                   const float* __restrict__ tensor_absmax, double* __restrict__ partial) {
   // rows between two first-stage flushes: every row adds 2*V terms to each half of a packed accumulator
   constexpr int kFlushRows = (kChainTerms / (2 * V)) > 0 ? (kChainTerms / (2 * V)) : 1;
+  // Programmatic dependent launch: the block is scheduled while the previous kernel of the stream
+  // drains and waits here for that kernel's results (result slots, per-tensor maxima, and whatever
+  // produced the weights).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const SweepBlock blk = blocks[blockIdx.x];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   __shared__ float smax2[2][kThreads / 32];
@@ -253,6 +258,8 @@ sweep_rows_kernel(const SweepSeg* __restrict__ segs, const SweepBlock* __restric
 __global__ void __launch_bounds__(kThreads)
 sweep_generic_kernel(const SweepSeg* __restrict__ segs, const SweepBlock* __restrict__ blocks, int per_tensor,
                      const float* __restrict__ tensor_absmax, int jlo, int jhi, double* __restrict__ partial) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const SweepBlock blk = blocks[blockIdx.x];
   const int lane = threadIdx.x & 31;
   __shared__ float smax[kThreads / 32];
@@ -310,6 +317,8 @@ sweep_generic_kernel(const SweepSeg* __restrict__ segs, const SweepBlock* __rest
 __global__ void __launch_bounds__(256)
 sweep_finalize_kernel(const double* __restrict__ partial, const TensorSlots* __restrict__ ts, int jlo, int nb,
                       double* __restrict__ sse, float* __restrict__ absmax, int write_absmax) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");     // the slots come from the kernels before
   __shared__ double sm[32][8];
   const int t = blockIdx.x;
   const int j = threadIdx.x & 7, g = threadIdx.x >> 3;
@@ -332,11 +341,28 @@ sweep_finalize_kernel(const double* __restrict__ partial, const TensorSlots* __r
   }
 }
 
+// Launch configuration with programmatic stream serialization: the kernel may start while its
+// predecessor in the stream drains; it orders itself with griddepcontrol.wait.
+cudaLaunchAttribute g_pdl_attr;
+inline cudaLaunchConfig_t pdl_config(int blocks, int threads, size_t smem, cudaStream_t st) {
+  g_pdl_attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  g_pdl_attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks);
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = &g_pdl_attr;
+  cfg.numAttrs = 1;
+  return cfg;
+}
+
 template <int V>
 void launch_rows(const SweepSeg* segs, const SweepBlock* blocks, int n_blocks, int per_tensor, const float* amax,
                  double* partial, cudaStream_t st) {
   constexpr size_t smem = (size_t)kRing * V * kThreads * sizeof(float4);
-  sweep_rows_kernel<V><<<n_blocks, kThreads, smem, st>>>(segs, blocks, per_tensor, amax, partial);
+  cudaLaunchConfig_t cfg = pdl_config(n_blocks, kThreads, smem, st);
+  cudaLaunchKernelEx(&cfg, sweep_rows_kernel<V>, segs, blocks, per_tensor, amax, partial);
 }
 
 template <int V>
@@ -451,7 +477,11 @@ int run_plan(Ctx* ctx, const Plan& P, const SweepSeg* segs, const SweepBlock* bl
     const SweepBlock* b = blocks + P.class_block0[c];
     prof_begin(ctx, 2, st);
     switch (c) {
-      case 0: sweep_generic_kernel<<<n, kThreads, 0, st>>>(segs, b, per_tensor, absmax, jlo, jhi, partial); break;
+      case 0: {
+        cudaLaunchConfig_t cfg = pdl_config(n, kThreads, 0, st);
+        cudaLaunchKernelEx(&cfg, sweep_generic_kernel, segs, b, per_tensor, (const float*)absmax, jlo, jhi, partial);
+        break;
+      }
       case 1: launch_rows<1>(segs, b, n, per_tensor, absmax, partial, st); break;
       case 2: launch_rows<2>(segs, b, n, per_tensor, absmax, partial, st); break;
       case 3: launch_rows<3>(segs, b, n, per_tensor, absmax, partial, st); break;
@@ -466,7 +496,10 @@ int run_plan(Ctx* ctx, const Plan& P, const SweepSeg* segs, const SweepBlock* bl
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return check_cuda(ctx, e, "sweep launch");
   }
-  sweep_finalize_kernel<<<n_tensors, 256, 0, st>>>(partial, slots, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
+  {
+    cudaLaunchConfig_t cfg = pdl_config(n_tensors, 256, 0, st);
+    cudaLaunchKernelEx(&cfg, sweep_finalize_kernel, (const double*)partial, slots, jlo, nb, sse, absmax, per_tensor ? 0 : 1);
+  }
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "sweep finalize launch");
 }
