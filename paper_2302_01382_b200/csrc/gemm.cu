@@ -9,9 +9,12 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=32 B per instruction)
 //               from shared-memory descriptors into one of two TMEM accumulator buffers
 //               (2 x 256 columns), and commits stage-release / accumulator-ready barriers.
-//   warps 2..17 epilogue: tcgen05.ld of the accumulator (one row per thread, 32 columns per
+//   warps 2..17 epilogue: tcgen05.ld of the accumulator (one row per thread, 16 or 32 columns per
 //               load), rescale, shortcut add, activation, stores of fp32 and/or the consumer's
-//               int8 / bf16 codes; overlaps the next tile's main loop.
+//               int8 / bf16 codes through shared-memory staging and TMA stores; overlaps the next
+//               tile's main loop.
+//   warps 18,19 (convolution launches only, 640 threads) gather the A tile of an implicit-GEMM
+//               convolution from the NHWC codes of the layer's input with cp.async.
 // Every mbarrier wait is bounded: after ~2 s it sets the context's error word and the CTA
 // leaves through the normal teardown (TMEM is freed).
 #include <cuda.h>
