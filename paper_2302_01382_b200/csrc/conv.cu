@@ -185,6 +185,60 @@ __global__ void __launch_bounds__(256) im2col_quantize_kernel(const float* __res
   }
 }
 
+
+// Inputs with few channels (the 3-channel stem): one block per output row (b, oh).  The kh input
+// rows the row's patches draw from are staged in shared memory with coalesced loads, zero-padded on
+// both sides (and zero where they fall outside the image), so building the patches needs no bounds
+// checks and no divisions: a table gives every k its offset (dy * row length + position in the
+// kernel row).  Consecutive threads write consecutive 8-element groups of an output row.
+template <bool BF16>
+__global__ void __launch_bounds__(256) im2col_rows_kernel(const float* __restrict__ src, ConvGeom g, float inv_scale, float qmax,
+                                                          void* __restrict__ q, int64_t ldq) {
+  extern __shared__ float srows[];                 // [kh][rowlen] then int koff[ldq]
+  const int rowlen = (g.W + 2 * g.pad) * g.C;
+  int* koff = reinterpret_cast<int*>(srows + g.kh * rowlen);
+  const int boh = blockIdx.x;
+  const int b = boh / g.OH, oh = boh - b * g.OH;
+  const float* img = src + (int64_t)b * g.H * g.WC;
+  for (int i = threadIdx.x; i < g.kh * rowlen; i += blockDim.x) {
+    const int dy = i / rowlen, p = i - dy * rowlen - g.pad * g.C;
+    const int ih = oh * g.stride - g.pad + dy;
+    srows[i] = (ih >= 0 && ih < g.H && p >= 0 && p < g.WC) ? __ldg(img + (int64_t)ih * g.WC + p) : 0.0f;
+  }
+  for (int k = threadIdx.x; k < (int)ldq; k += blockDim.x) {
+    const int dy = k / g.kwC;
+    koff[k] = k < g.K ? dy * rowlen + (k - dy * g.kwC) : -1;
+  }
+  __syncthreads();
+  const int gpr = (int)(ldq >> 3);
+  for (int it = threadIdx.x; it < g.OW * gpr; it += blockDim.x) {
+    const int ow = it / gpr, k0 = (it - ow * gpr) << 3;
+    const int base = ow * g.stride * g.C;
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int o = koff[k0 + j];
+      v[j] = o >= 0 ? srows[o + base] : 0.0f;
+    }
+    const int64_t row = (int64_t)boh * g.OW + ow;
+    if (BF16) {
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        w[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(q) + row * ldq + k0) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+      const uint32_t lo = conv_pack4(conv_code(v[0], inv_scale, qmax), conv_code(v[1], inv_scale, qmax),
+                                     conv_code(v[2], inv_scale, qmax), conv_code(v[3], inv_scale, qmax));
+      const uint32_t hi = conv_pack4(conv_code(v[4], inv_scale, qmax), conv_code(v[5], inv_scale, qmax),
+                                     conv_code(v[6], inv_scale, qmax), conv_code(v[7], inv_scale, qmax));
+      *reinterpret_cast<uint2*>(reinterpret_cast<int8_t*>(q) + row * ldq + k0) = make_uint2(lo, hi);
+    }
+  }
+}
+
 int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, int C, int kh, int kw, int stride,
                            int pad, float inv_scale, int bits, void* q, int64_t ldq, cudaStream_t st) {
   ConvGeom g;
@@ -198,6 +252,15 @@ int launch_im2col_quantize(Ctx* ctx, const float* src, int64_t B, int H, int W, 
   if (rows == 0) return QCFG_OK;
   if (B * g.OH > 0x7fffffff || (int64_t)W * C > 0x7fffffff) return set_error(ctx, QCFG_ESHAPE, "im2col: image too large");
   const int vec = (C % 8 == 0 && (uintptr_t)src % 16 == 0) ? 1 : 0;
+  const size_t rows_smem = ((size_t)kh * (W + 2 * pad) * C + (size_t)ldq) * 4;
+  if (!vec && rows_smem <= 48 * 1024) {          // few channels: the row-staged kernel
+    prof_begin(ctx, 2, st);
+    if (bits == 16) im2col_rows_kernel<true><<<(unsigned)(B * g.OH), 256, rows_smem, st>>>(src, g, 1.0f, 0.0f, q, ldq);
+    else im2col_rows_kernel<false><<<(unsigned)(B * g.OH), 256, rows_smem, st>>>(src, g, inv_scale, qmax_of(bits), q, ldq);
+    prof_end(ctx, 2, 0.0, st);
+    count_launch(ctx);
+    return check_cuda(ctx, cudaGetLastError(), "im2col launch");
+  }
   const int gpr = (int)(ldq >> 3);
   const int bx = gpr >= 24 ? 32 : (gpr >= 12 ? 16 : 8);
   const int by = 256 / bx;
