@@ -13,11 +13,20 @@ __global__ void __launch_bounds__(256) maxpool3s2_kernel(const float* __restrict
   const int64_t total = B * OH * OW * cg;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
-  const int c = (int)(idx % cg);
-  int64_t t = idx / cg;
-  const int ow = (int)(t % OW); t /= OW;
-  const int oh = (int)(t % OH);
-  const int64_t b = t / OH;
+  int c, ow, oh;
+  int64_t b;
+  if (total <= 0x7fffffff) {            // 32-bit index arithmetic (64-bit divisions cost an order of magnitude more)
+    const unsigned i = (unsigned)idx, t1 = i / (unsigned)cg, t2 = t1 / (unsigned)OW;
+    c = (int)(i - t1 * cg); ow = (int)(t1 - t2 * OW);
+    const unsigned t3 = t2 / (unsigned)OH;
+    oh = (int)(t2 - t3 * OH); b = t3;
+  } else {
+    c = (int)(idx % cg);
+    int64_t t = idx / cg;
+    ow = (int)(t % OW); t /= OW;
+    oh = (int)(t % OH);
+    b = t / OH;
+  }
   const float ninf = __int_as_float(0xff800000);
   float4 m = make_float4(ninf, ninf, ninf, ninf);
 #pragma unroll
