@@ -219,6 +219,7 @@ struct Model {
   bool calibrated = false;
   bool evaluated = false;
   DevBuf act_absmax_dev;           // fp32 [n_layers], filled by calibration
+  std::vector<int> calib_same_as;  // layer whose calibrated maximum layer l shares (same input tensor), or -1
   DevBuf search_ref, search_out, search_partial;   // buffers of the search drivers
   DevBuf noise_codes, noise_amax;                  // perturbed bf16 weights of one layer and its max|w|
   DevBuf adj_gs, adj_gt, adj_qxt, adj_qwt, adj_dx, adj_dw, adj_colsum, adj_dscal;   // scale adjustment temporaries
@@ -431,9 +432,14 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       }
       const int64_t width = d.kh > 0 ? d.in_c : d.k_in;       // columns of the tensor that is calibrated
       const float* tp = sp + (d.kh > 0 ? 0 : d.src_col0);
-      if (calibrate) {
+      // calibration: a tensor that is also turned into a 16-bit row operand below gets its range
+      // from that same launch; one that an earlier layer already read takes that layer's value
+      bool range_pending = calibrate;
+      if (calibrate) M->calib_same_as[l] = -1;
+      if (calibrate && !(direct && !S.implicit)) {
         rc = launch_absmax(ctx, tp, srows, width, sld, QCFG_PER_TENSOR, (float*)M->act_absmax_dev.p + l, st);
         if (rc) return rc;
+        range_pending = false;
       }
       // reuse the codes of an earlier layer that reads the same input with the same grid
       int share = -1;
@@ -445,6 +451,15 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       }
       if (share >= 0) {
         S.a_ptr = M->L[share].a_ptr;
+        if (range_pending) {
+          // same tensor, same maximum; a chain of sharers ends at the layer that measured it
+          if (M->calib_same_as[share] >= 0 || (reads_rows_directly(M->L[share].d) && !M->L[share].implicit)) {
+            M->calib_same_as[l] = M->calib_same_as[share] >= 0 ? M->calib_same_as[share] : share;
+          } else {
+            rc = launch_absmax(ctx, tp, srows, width, sld, QCFG_PER_TENSOR, (float*)M->act_absmax_dev.p + l, st);
+            if (rc) return rc;
+          }
+        }
       } else {
         rc = S.abuf.ensure(ctx, (size_t)(S.implicit ? srows * d.in_c : S.rows * S.ldk) * 2);
         if (rc) return rc;
@@ -453,7 +468,8 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
         if (S.implicit)      // the input tensor's own codes, NHWC; the GEMM gathers the patches
           rc = launch_quantize(ctx, sp, srows, d.in_c, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, d.in_c, st);
         else if (direct)
-          rc = launch_quantize(ctx, tp, S.rows, d.k_in, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st);
+          rc = launch_quantize(ctx, tp, S.rows, d.k_in, sld, nullptr, inv, QCFG_PER_TENSOR, b, S.abuf.p, S.ldk, st,
+                               range_pending ? (float*)M->act_absmax_dev.p + l : nullptr);
         else
           rc = launch_im2col_quantize(ctx, sp, m, d.in_h, d.in_w, d.in_c, d.kh, d.kw, d.stride, d.pad, inv, b, S.abuf.p, S.ldk, st);
         if (rc) return rc;
@@ -827,6 +843,7 @@ int qcfg_model_create(qcfg_ctx* ctx, const qcfg_layer* layers, int32_t n_layers,
   Model* M = &h->m;
   M->ctx = c;
   M->L.resize(n_layers);
+  M->calib_same_as.assign(n_layers, -1);
   int rc = M->act_absmax_dev.ensure(c, (size_t)n_layers * 4);
   for (int l = 0; l < n_layers && !rc; ++l) {
     LayerState& S = M->L[l];
@@ -875,6 +892,8 @@ int qcfg_calibrate_model(qcfg_ctx* ctx, qcfg_model* model, const float* x_dev, i
   rc = check_cuda(c, cudaMemcpyAsync(host.data(), M->act_absmax_dev.p, host.size() * 4, cudaMemcpyDeviceToHost, st), "calibration table copy");
   if (!rc) rc = qcfg_sync_status(ctx, stream);
   if (rc) return rc;
+  for (size_t l = 0; l < host.size(); ++l)
+    if (M->calib_same_as[l] >= 0) host[l] = host[(size_t)M->calib_same_as[l]];
   for (size_t l = 0; l < host.size(); ++l)
     if (!std::isfinite(host[l])) return set_error(c, QCFG_ENONFINITE, "layer %zu: calibrated input maximum is not finite", l);
   for (size_t l = 0; l < host.size(); ++l) M->L[l].act_absmax = host[l];

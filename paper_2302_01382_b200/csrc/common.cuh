@@ -42,10 +42,11 @@ int launch_absmax(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t 
                   int granularity, float* absmax, cudaStream_t st);
 int launch_scales(Ctx* ctx, const float* absmax, int64_t n, int bits, float* scale,
                   float* inv_scale, cudaStream_t st);
-// inv_scale_ptr (device) or, when null, inv_scale_val for the whole tensor
+// inv_scale_ptr (device) or, when null, inv_scale_val for the whole tensor; with `absmax` set
+// (16-bit only) the same launch also leaves max |x| of the tensor there
 int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t ld,
                     const float* inv_scale_ptr, float inv_scale_val, int granularity, int bits,
-                    void* q, int64_t ldq, cudaStream_t st);
+                    void* q, int64_t ldq, cudaStream_t st, float* absmax = nullptr);
 
 int launch_perturb_bf16(Ctx* ctx, const float* w, const float* nu, const float* amax_dev, float lambda, int64_t rows,
                         int64_t cols, void* q, int64_t ldq, cudaStream_t st);

@@ -148,51 +148,79 @@ __device__ __forceinline__ int quant_code(float x, float inv_scale, float qmax) 
   return __float2int_rn(t);
 }
 
-// Each thread produces 8 consecutive output elements of one row.
+// Each thread produces 8 consecutive output elements of one row.  With `amax` set the launch also
+// folds max |x| of everything it read into *amax (bit patterns, so exact in any order): calibration
+// reads each activation tensor once for both its range and its 16-bit operand.
 template <bool BF16>
 __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__ x, int64_t rows, int64_t cols,
                                                        int64_t ld, const float* __restrict__ inv_scale_ptr,
                                                        float inv_scale_val, int per_row, float qmax,
-                                                       void* __restrict__ q, int64_t ldq, int vec) {
+                                                       void* __restrict__ q, int64_t ldq, int vec,
+                                                       unsigned* __restrict__ amax) {
   const int64_t gpr = ldq >> 3;  // groups of 8 per output row
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * gpr) return;
-  const int64_t row = idx / gpr;
-  const int64_t c0 = (idx - row * gpr) << 3;
-  float v[8];
-  const float* p = x + row * ld + c0;
-  if (vec && c0 + 8 <= cols) {
-    float4 a = __ldg(reinterpret_cast<const float4*>(p));
-    float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-  } else {
+  unsigned m = 0;
+  if (idx < rows * gpr) {
+    const int64_t row = idx / gpr;
+    const int64_t c0 = (idx - row * gpr) << 3;
+    float v[8];
+    const float* p = x + row * ld + c0;
+    if (vec && c0 + 8 <= cols) {
+      float4 a = __ldg(reinterpret_cast<const float4*>(p));
+      float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = (c0 + j < cols) ? __ldg(p + j) : 0.0f;
+      for (int j = 0; j < 8; ++j) v[j] = (c0 + j < cols) ? __ldg(p + j) : 0.0f;
+    }
+    if (BF16) {
+      if (amax) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          unsigned a = abs_bits(v[j]);
+          m = m > a ? m : a;
+        }
+      }
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        o[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(q) + row * ldq + c0) =
+          make_uint4(o[0], o[1], o[2], o[3]);
+    } else {
+      float inv = inv_scale_ptr ? (per_row ? __ldg(inv_scale_ptr + row) : __ldg(inv_scale_ptr)) : inv_scale_val;
+      uint32_t lo = 0, hi = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        lo |= (uint32_t)(quant_code(v[j], inv, qmax) & 0xff) << (8 * j);
+        hi |= (uint32_t)(quant_code(v[j + 4], inv, qmax) & 0xff) << (8 * j);
+      }
+      *reinterpret_cast<uint2*>(reinterpret_cast<int8_t*>(q) + row * ldq + c0) = make_uint2(lo, hi);
+    }
   }
-  if (BF16) {
-    uint32_t o[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-      o[j] = *reinterpret_cast<uint32_t*>(&h);
+  if (BF16 && amax) {       // uniform over the block: no thread has left
+    m = warp_max_u(m);
+    __shared__ unsigned sm[8];
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      m = threadIdx.x < 8 ? sm[threadIdx.x] : 0u;
+      m = warp_max_u(m);
+      if (threadIdx.x == 0 && m) atomicMax(amax, m);
     }
-    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(q) + row * ldq + c0) =
-        make_uint4(o[0], o[1], o[2], o[3]);
-  } else {
-    float inv = inv_scale_ptr ? (per_row ? __ldg(inv_scale_ptr + row) : __ldg(inv_scale_ptr)) : inv_scale_val;
-    uint32_t lo = 0, hi = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      lo |= (uint32_t)(quant_code(v[j], inv, qmax) & 0xff) << (8 * j);
-      hi |= (uint32_t)(quant_code(v[j + 4], inv, qmax) & 0xff) << (8 * j);
-    }
-    *reinterpret_cast<uint2*>(reinterpret_cast<int8_t*>(q) + row * ldq + c0) = make_uint2(lo, hi);
   }
 }
 
 int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_t ld,
                     const float* inv_scale_ptr, float inv_scale_val, int granularity, int bits, void* q,
-                    int64_t ldq, cudaStream_t st) {
+                    int64_t ldq, cudaStream_t st, float* absmax) {
+  if (absmax) {
+    if (bits != 16) return set_error(ctx, QCFG_EINVAL, "quantize: the fused range is computed with 16-bit operands only");
+    cudaError_t e = cudaMemsetAsync(absmax, 0, sizeof(float), st);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "memset absmax");
+  }
   if (rows == 0 || ldq == 0) return QCFG_OK;
   // vector loads need every row start and every group start 16-byte aligned
   const int vec = ((uintptr_t)x % 16 == 0 && ld % 4 == 0) ? 1 : 0;
@@ -200,12 +228,13 @@ int launch_quantize(Ctx* ctx, const float* x, int64_t rows, int64_t cols, int64_
   const unsigned blocks = (unsigned)((total + 255) / 256);
   if (bits == 16) {
     prof_begin(ctx, 2, st);
-    quantize_kernel<true><<<blocks, 256, 0, st>>>(x, rows, cols, ld, nullptr, 1.0f, 0, 0.0f, q, ldq, vec);
+    quantize_kernel<true><<<blocks, 256, 0, st>>>(x, rows, cols, ld, nullptr, 1.0f, 0, 0.0f, q, ldq, vec,
+                                                  reinterpret_cast<unsigned*>(absmax));
     prof_end(ctx, 2, 0.0, st);
   } else {
     prof_begin(ctx, 2, st);
     quantize_kernel<false><<<blocks, 256, 0, st>>>(x, rows, cols, ld, inv_scale_ptr, inv_scale_val,
-                                                   granularity == QCFG_PER_ROW, qmax_of(bits), q, ldq, vec);
+                                                   granularity == QCFG_PER_ROW, qmax_of(bits), q, ldq, vec, nullptr);
     prof_end(ctx, 2, 0.0, st);
   }
   count_launch(ctx);
