@@ -37,7 +37,7 @@ TOKENS = 32 * 384
 WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
 # DRAM bytes (read + write) per int8 GEMM launch from the ncu capture summarised in
 # profiles/gemm_int8_bert_base_block.md; set to None whenever the GEMM kernel changes.
-GEMM_TRAFFIC_BYTES = 27.3e6
+GEMM_TRAFFIC_BYTES = None
 DATASHEET_INT8_TOPS = 4500.0      # B200 dense int8, vendor datasheet (an outside figure)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -521,7 +521,7 @@ def run_gpu(args):
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": clocks, "gpu_launches": int(launches),
             "host": {"enqueue_ms_per_eval": host_enqueue_ms, "device_ms_per_eval": ms_total / args.steps / N_EVALS,
-                     "note": "host time of one qcfg_eval_config call (planning, tensor maps, 48 launches) against the device time it hides behind"},
+                     "note": "host time of one qcfg_eval_config call (planning, tensor maps, 48 GEMM records in 7 chained launches) against the device time it hides behind"},
             "e2e": e2e, "launches_before_timed": int(launches0),
             "roofline": {"kernel": "gemm_kernel<int8>", "bound": "tensor", "achieved": achieved, "peak": sustained2,
                          "unit": "TOP/s", "frac": achieved / sustained2,
@@ -532,14 +532,16 @@ def run_gpu(args):
                          "launches": int(g_n), "avg_launch_us": 1e3 * g_ms / max(g_n, 1),
                          "kernel_ms_per_step": g_ms / args.steps, "bf16_kernel_ms_per_step": b_ms / args.steps,
                          "traffic": GEMM_TRAFFIC_BYTES,
-                         "traffic_source": "ncu dram bytes per launch, mean of the four GEMM launches (q/k/v grouped, o, ffn1, ffn2) of one block at 12288 tokens",
+                         "traffic_source": "none: the kernel changed after the last ncu capture" if GEMM_TRAFFIC_BYTES is None else
+                                           "ncu dram bytes per launch (a chain of layers' GEMMs at 12288 tokens)",
                          "how": "the timed pass that gives `value`: every CTA folds %globaltimer after its wait for the "
-                                "previous kernel and at its end into the launch's slot; duration = last end - first start",
+                                "previous kernel and at its end into the launch's slot; duration = last end - first start; "
+                                "a launch is a chain of up to seven consecutive layers' GEMMs",
                          "event_pass": {"int8_gemm_avg_launch_us": 1e3 * eg_ms / max(eg_n, 1),
                                         "tops": eg_ops / (eg_ms * 1e-3) / 1e12 if eg_ms else None,
                                         "share_of_kernel_time": eg_ms / max(eg_ms + eb_ms + eo_ms, 1e-9),
                                         "step_ms": instrumented_ms,
-                                        "how": "one extra step with CUDA events around every launch (launches serialised)"}},
+                                        "how": "one extra step with CUDA events around every launch (one launch per GEMM, serialised, no chains)"}},
             "sweep": {"gbs": sweep_gbs, "ms": sweep_ms, "bytes": sweep_bytes, "hbm_peak_gbs": peaks["hbm_gbs"],
                       "frac": sweep_gbs / peaks["hbm_gbs"], "peak_source": peaks["_source"],
                       "sustained": {"calls": n_long, "gbs": sweep_long_gbs, "ms": sweep_long_ms, "sm_mhz": sweep_clock,

@@ -24,7 +24,7 @@ EINVAL, EBITS, ESHAPE, EALIGN, ENOMEM, ENONFINITE, EARCH, ECUDA, ETIMEOUT = rang
 ESTATE = 11
 
 EXPORTS = ["qcfg_create", "qcfg_destroy", "qcfg_sync_status", "qcfg_selftest_wait_timeout", "qcfg_last_error", "qcfg_launch_count",
-           "qcfg_set_fusion", "qcfg_set_pair_tiles", "qcfg_set_grouping", "qcfg_set_prefix_reuse", "qcfg_set_implicit_conv", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
+           "qcfg_set_fusion", "qcfg_set_pair_tiles", "qcfg_set_grouping", "qcfg_set_prefix_reuse", "qcfg_set_implicit_conv", "qcfg_set_gemm_chains", "qcfg_profile_enable", "qcfg_profile_read", "qcfg_calibrate", "qcfg_scales_from_absmax", "qcfg_quantize",
            "qcfg_quant_error_sweep", "qcfg_quant_error_sweep_static", "qcfg_gemm_i8", "qcfg_gemm_i8_requant", "qcfg_gemm_bf16", "qcfg_model_create",
            "qcfg_model_destroy", "qcfg_calibrate_model", "qcfg_model_act_absmax",
            "qcfg_model_weight_absmax", "qcfg_eval_config", "qcfg_latency_table", "qcfg_config_cost", "qcfg_noise_sensitivity", "qcfg_search", "qcfg_adjust_scales", "qcfg_scale_gradients", "qcfg_model_scales",
@@ -68,6 +68,7 @@ def load_library() -> C.CDLL:
         "qcfg_set_grouping": [vp, ci],
         "qcfg_set_prefix_reuse": [vp, ci],
         "qcfg_set_implicit_conv": [vp, ci],
+        "qcfg_set_gemm_chains": [vp, ci],
         "qcfg_profile_enable": [vp, ci],
         "qcfg_profile_read": [vp, ci, C.POINTER(C.c_double), C.POINTER(i64), C.POINTER(C.c_double), ci],
         "qcfg_calibrate": [vp, vp, i64, i64, i64, ci, vp, vp],
@@ -172,6 +173,9 @@ class Context:
 
     def set_implicit_conv(self, enabled: bool):
         self._check(self.lib.qcfg_set_implicit_conv(self.h, int(enabled)))
+
+    def set_gemm_chains(self, enabled: bool):
+        self._check(self.lib.qcfg_set_gemm_chains(self.h, int(enabled)))
 
     def set_pair_tiles(self, enabled: bool):
         self._check(self.lib.qcfg_set_pair_tiles(self.h, int(enabled)))

@@ -23,6 +23,8 @@ struct Ctx {
   int pair = 1;                     // two-CTA GEMM tiles where they apply
   int group = 1;                    // independent GEMMs of equal shape share a launch
   int implicit = 1;                 // convolutions gather their patches inside the GEMM (no im2col matrix)
+  int chain = 1;                    // consecutive GEMMs of a forward pass share one cooperative launch
+  void* chain_state = nullptr;      // owned by gemm.cu
   int reuse = 0;                    // evaluations restart at the first layer whose bit width changed
   int64_t epoch = 0;                // bumped by every switch that changes which buffers hold what
   int pair_clusters[2] = {0, 0};
@@ -111,6 +113,9 @@ int sm_count(Ctx* ctx) { return ctx->sms; }
 bool ctx_pair_enabled(Ctx* ctx) { return ctx->pair != 0; }
 int* pair_cluster_cache(Ctx* ctx) { return ctx->pair_clusters; }
 int device_of(Ctx* ctx) { return ctx->device; }
+void*& chain_slot(Ctx* ctx) { return ctx->chain_state; }
+bool ctx_chain_enabled(Ctx* ctx) { return ctx->chain != 0; }
+int prof_mode(Ctx* ctx) { return ctx->prof; }
 
 int set_error(Ctx* ctx, int code, const char* fmt, ...) {
   if (ctx) {
@@ -168,7 +173,7 @@ struct DevBuf {
   size_t bytes = 0;
   int ensure(Ctx* ctx, size_t want) {
     if (want <= bytes) return QCFG_OK;
-    if (p) { cudaDeviceSynchronize(); cudaFree(p); p = nullptr; bytes = 0; }
+    if (p) { gemm_chain_flush(ctx); cudaDeviceSynchronize(); cudaFree(p); p = nullptr; bytes = 0; }   // nothing deferred may still name p
     cudaError_t e = cudaMalloc(&p, want);
     if (e != cudaSuccess) { cudaGetLastError(); p = nullptr; return set_error(ctx, QCFG_ENOMEM, "cudaMalloc of %zu bytes failed", want); }
     bytes = want;
@@ -262,7 +267,8 @@ int ensure_weight_codes(Ctx* ctx, LayerState& S, int bits, cudaStream_t st) {
   WeightCodes& W = S.wc[bits];
   if (W.ready) return QCFG_OK;
   const int64_t n = S.d.n_out, k = S.d.k_in;
-  int rc = W.codes.ensure(ctx, (size_t)(n * S.ldk) * (bits == 16 ? 2 : 1));
+  int rc = gemm_chain_flush(ctx);      // other kernels follow on the stream
+  if (!rc) rc = W.codes.ensure(ctx, (size_t)(n * S.ldk) * (bits == 16 ? 2 : 1));
   if (rc) return rc;
   if (bits == 16) {
     rc = launch_quantize(ctx, S.d.w_dev, n, k, k, nullptr, 1.0f, QCFG_PER_ROW, 16, W.codes.p, S.ldk, st);
@@ -319,6 +325,12 @@ void reset_adjusted_scales(Model* M) {
 int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t x_ld, int64_t m,
             float* const* y_dev, bool calibrate, cudaStream_t st, cudaEvent_t* layer_ev = nullptr) {
   const int n = (int)M->L.size();
+  // GEMM launches of this pass may be collected into chains; every way out closes the chain
+  struct ChainScope {
+    Ctx* c; bool armed;
+    ~ChainScope() { if (armed) gemm_chain_close(c); }
+  } scope{ctx, true};
+  gemm_chain_open(ctx);
   // Prefix reuse: the layers' buffers still hold the previous evaluation (same input, same rows).
   // A layer is recomputed ("dirty") when its bit width changed, when the caller wants its output,
   // or when a layer it reads was recomputed; everything else keeps its buffers and launches
@@ -385,10 +397,16 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     int rc = ensure_weight_codes(ctx, S, b, st);
     if (rc) return rc;
     // optional per-layer timing: everything this layer launches (operand preparation and GEMM)
-    if (layer_ev && cudaEventRecord(layer_ev[2 * l], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
+    if (layer_ev) {
+      rc = gemm_chain_flush(ctx);
+      if (rc) return rc;
+      if (cudaEventRecord(layer_ev[2 * l], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
+    }
 
     // ---- GEMM input codes
     if (!S.a_ready) {
+      rc = gemm_chain_flush(ctx);      // the kernels below follow the deferred GEMMs on the stream
+      if (rc) return rc;
       // the fp32 tensor this layer reads: [srows x sld], NHWC for the convolutional table
       const float* sp; int64_t sld, srows;
       if (d.src < 0) {
@@ -555,9 +573,16 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       rc = launch_gemm(ctx, g, st);
       if (rc) return rc;
     }
-    if (layer_ev && cudaEventRecord(layer_ev[2 * l + 1], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
+    if (layer_ev) {
+      rc = gemm_chain_flush(ctx);
+      if (rc) return rc;
+      if (cudaEventRecord(layer_ev[2 * l + 1], st) != cudaSuccess) return check_cuda(ctx, cudaGetLastError(), "event record");
+    }
   }
-  const int frc = flush();
+  int frc = flush();
+  const int crc = gemm_chain_close(ctx);
+  scope.armed = false;
+  if (frc == QCFG_OK) frc = crc;
   if (frc == QCFG_OK && !calibrate && !layer_ev) {
     M->reuse_valid = true; M->reuse_x = x_dev; M->reuse_m = m; M->reuse_epoch = ctx->epoch;
   }
@@ -593,7 +618,7 @@ int qcfg_create(qcfg_ctx** out, int device) {
   }
   int rc = gemm_init(&h->c);
   if (!rc) rc = sweep_init(&h->c);
-  if (rc) { cudaFree(h->c.err_dev); delete h; return rc; }
+  if (rc) { gemm_destroy(&h->c); cudaFree(h->c.err_dev); delete h; return rc; }
   *out = h;
   return QCFG_OK;
 }
@@ -605,6 +630,7 @@ int qcfg_destroy(qcfg_ctx* ctx) {
   if (ctx->c.scratch_buf) cudaFree(ctx->c.scratch_buf);
   if (ctx->c.stamp_dev) cudaFree(ctx->c.stamp_dev);
   if (ctx->c.err_dev) cudaFree(ctx->c.err_dev);
+  gemm_destroy(&ctx->c);
   delete ctx;
   return QCFG_OK;
 }
@@ -619,6 +645,7 @@ int qcfg_sync_status(qcfg_ctx* ctx, void* stream) {
   if (e != cudaSuccess) return check_cuda(c, e, "error word read");
   if (w) {
     cudaMemset(c->err_dev, 0, sizeof(w));
+    gemm_chain_reset(c);
     if (w & ERR_TIMEOUT) return set_error(c, QCFG_ETIMEOUT, "a bounded device-side wait gave up");
     if (w & ERR_NONFINITE) return set_error(c, QCFG_ENONFINITE, "non-finite value found on the device");
   }
@@ -689,6 +716,11 @@ int qcfg_set_implicit_conv(qcfg_ctx* ctx, int enabled) {
   if (!ctx) return QCFG_EINVAL;
   ctx->c.implicit = enabled ? 1 : 0;
   ctx->c.epoch++;
+  return QCFG_OK;
+}
+int qcfg_set_gemm_chains(qcfg_ctx* ctx, int enabled) {
+  if (!ctx) return QCFG_EINVAL;
+  ctx->c.chain = enabled ? 1 : 0;
   return QCFG_OK;
 }
 int qcfg_set_prefix_reuse(qcfg_ctx* ctx, int enabled) {

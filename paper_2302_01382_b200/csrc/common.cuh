@@ -23,6 +23,9 @@ int sm_count(Ctx* ctx);
 bool ctx_pair_enabled(Ctx* ctx);
 int* pair_cluster_cache(Ctx* ctx);   // [2]: resident CTA pairs of the int8 / bf16 pair kernels, 0 = not yet queried
 int device_of(Ctx* ctx);
+void*& chain_slot(Ctx* ctx);         // gemm.cu's per-context state
+bool ctx_chain_enabled(Ctx* ctx);
+int prof_mode(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);
 // grows (never shrinks) a host buffer owned by the context; returns nullptr on failure
@@ -127,6 +130,14 @@ int launch_gemm(Ctx* ctx, const GemmArgs& g, cudaStream_t st);
 bool gemm_groupable(const GemmArgs& a, const GemmArgs& b);
 int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st);
 int gemm_init(Ctx* ctx);   // resolves the tensor-map encoder, sets smem attributes
+void gemm_destroy(Ctx* ctx);
+// Chains: while one is open, GEMM launches that qualify (pair flavour, 256-column tiles, no
+// gather) are collected and go to the device as one launch at the next flush; anything else that
+// is put on the stream in between must flush first.
+void gemm_chain_open(Ctx* ctx);
+int gemm_chain_flush(Ctx* ctx);
+int gemm_chain_close(Ctx* ctx);
+int gemm_chain_reset(Ctx* ctx);
 int launch_wait_timeout(Ctx* ctx, uint64_t limit_ns, cudaStream_t st);
 
 // ----- small device helpers -----------------------------------------------------------

@@ -21,6 +21,7 @@
 
 #include <cstring>
 #include <mutex>
+#include <new>
 #include <unordered_map>
 
 #include "common.cuh"
@@ -85,6 +86,7 @@ struct ConvDesc {
   int64_t img_bytes;          // bytes of one image (H * W * C * esz)
   const uint8_t* src;
 };
+constexpr int kMaxDeps = 4;
 struct GemmParams {
   int32_t m, k_blocks, bn, tiles_m, tiles_n, stages, is_bf16;   // tiles_n: column tiles of all groups together
   int32_t epi_bytes;          // staging bytes per epilogue warp (2048 or 4096)
@@ -93,7 +95,22 @@ struct GemmParams {
   unsigned* err;
   unsigned long long* stamp;  // optional [2]: earliest start / latest end of the launch's CTAs (%globaltimer, ns)
   ConvDesc conv;              // conv.on: A comes from the gather warps (single-group launches only)
+  // chains: records of the same launch whose output rows this record reads (-1: none), and
+  // whether a later record of the launch reads this one's
+  int32_t deps[kMaxDeps];
+  int32_t signal;
 };
+// What one launch gets: one record, or a chain of them (see the kernel).
+constexpr int kChainMax = 7;
+struct Rec { AllMaps maps; GemmParams p; };
+template <int N> struct LaunchArgs {
+  Rec rec[N];
+  int32_t n;             // records in use
+  int32_t total_tiles;   // tiles of all records together
+  int32_t flag_stride;   // counters per record (two per row tile: one per CTA of the pair)
+  unsigned* flags;       // [n x flag_stride], zero when the launch starts
+};
+static_assert(sizeof(LaunchArgs<kChainMax>) <= 32764, "kernel parameters are limited to 32764 bytes");
 
 // ---------------------------------------------------------------------------- PTX wrappers
 
@@ -133,6 +150,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       uint64_t now = global_timer();
       if (t0 == 0) t0 = now;
       else if (now - t0 > limit_ns) {
+        atomicOr(err, ERR_TIMEOUT);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+// Chains: waits until a counter of finished tiles has reached `need`.  Bounded like every other wait.
+__device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, volatile int* abort_flag, unsigned* err) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v >= need) return true;
+    if ((it & 63u) == 0) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
         atomicOr(err, ERR_TIMEOUT);
         *abort_flag = 1;
         return false;
@@ -408,10 +445,13 @@ __device__ __forceinline__ float2 code_words2(float2 y, float2 inv2, float qmax)
 // written by one TMA store.  Otherwise the fp32 matrix, each 32 x 32 block staged in 128-byte
 // rows (128B swizzle), one TMA store per block; the single staging slot is reused once the
 // previous store has read it.
+// done_bar (chains, else 0): barrier to arrive on once the stores this warp issued for its previous
+// tile have completed; that is checked just before this tile's first store, most of an epilogue
+// after they were issued.
 template <bool BF16, bool PAIR, bool CODES>
 __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUtensorMap* fmap, uint32_t tbase,
                                                    const float* cs, uint32_t stage, int row0, int col0, int lane,
-                                                   uint32_t tempty_bar) {
+                                                   uint32_t tempty_bar, uint32_t done_bar) {
   const int act = G.act;
   const float qmax = G.outs[2].qmax;
   const float2 inv2 = make_float2(G.outs[2].inv_scale, G.outs[2].inv_scale);
@@ -460,13 +500,25 @@ __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUt
     if (!CODES) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0 && col0 + 32 * h < G.n) tma_store_2d(fmap, stage, col0 + 32 * h, row0);
+      if (lane == 0) {
+        if (h == 0 && done_bar) {
+          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+          mbar_arrive(done_bar);
+        }
+        if (col0 + 32 * h < G.n) tma_store_2d(fmap, stage, col0 + 32 * h, row0);
+      }
     }
   }
   if (CODES) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0) tma_store_2d(fmap, stage, col0, row0);
+    if (lane == 0) {
+      if (done_bar) {
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        mbar_arrive(done_bar);
+      }
+      tma_store_2d(fmap, stage, col0, row0);
+    }
   }
 }
 
@@ -494,11 +546,12 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
       y[i] = __fmul_rn((float)(int32_t)v[i], __shfl_sync(0xffffffffu, cs_lane, i));
   }
   if (p.residual && row_ok) {
+    // read through L2: in a chain another SM may have written the shortcut earlier in this launch
     const float* r = p.residual + row * p.ldr + col0;
     if (full && (p.ldr & 3) == 0 && (((uintptr_t)p.residual) & 15) == 0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        float4 r4 = __ldg(reinterpret_cast<const float4*>(r) + i);
+        float4 r4 = __ldcg(reinterpret_cast<const float4*>(r) + i);
         y[4 * i + 0] = __fadd_rn(y[4 * i + 0], r4.x);
         y[4 * i + 1] = __fadd_rn(y[4 * i + 1], r4.y);
         y[4 * i + 2] = __fadd_rn(y[4 * i + 2], r4.z);
@@ -506,7 +559,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
       }
     } else {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) if (i < ncols) y[i] = __fadd_rn(y[i], __ldg(r + i));
+      for (int i = 0; i < 32; ++i) if (i < ncols) y[i] = __fadd_rn(y[i], __ldcg(r + i));
     }
   }
   if (p.act == QCFG_ACT_RELU) {
@@ -546,9 +599,23 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
 
 // ---------------------------------------------------------------------------- the kernel
 
-template <bool BF16, bool PAIR, bool GROUPED>
+// One launch runs one GEMM record or, in the CHAIN flavour, up to kChainMax records one after the
+// other: consecutive layers of a model, each reading what an earlier one wrote.  The tiles of all
+// records form one sequence (record after record, column tile fastest inside a record) that the
+// CTA pairs deal out round-robin, so a pair that runs out of tiles of one record goes on with the
+// next: no pipeline fill and drain, no idle last round and no kernel boundary between layers.
+// A tile may start when the row tiles it reads are complete: every finished tile adds one to a
+// counter of its (record, row tile, CTA rank), a warp of its own does that once the tile's stores
+// have completed, and the producer warp waits for the counters of the records its record names.
+// Waits only ever point at earlier tiles of the sequence and the launch is cooperative (all CTAs
+// resident), so the first unfinished tile can always proceed.  The records of a chain share tile
+// shape, operand type, stage count, staging size, rows and grid.
+template <bool BF16, bool PAIR, bool GROUPED, bool CHAIN>
 __global__ void __launch_bounds__(kGemmThreadsConv, 1)
-gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmParams p) {
+gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
+  const GemmParams& p = L.rec[0].p;        // what all records of the launch have in common is read here
+  const GemmParams* q = &L.rec[0].p;       // the record this thread's role is working on
+  const AllMaps* mp = &L.rec[0].maps;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the 128B swizzle atoms
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -570,20 +637,38 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   const uint32_t stage_bytes = (uint32_t)(BM + b_rows) * kStageKBytes;
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
   const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16;
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const uint32_t done0 = tempty0 + 16;           // chains: done[4], the epilogue warps' stores of a tile have completed
   const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // first tile of this CTA (pair)
   const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int rows_per_tile = PAIR ? 2 * BM : BM;
   // group of a column tile (a single-GEMM launch has only group 0, known at compile time)
   auto group_of = [&](int tn) -> int {
-    return GROUPED ? (int)(tn >= p.grp[1].tn_begin) + (int)(tn >= p.grp[2].tn_begin) : 0;
+    return GROUPED ? (int)(tn >= q->grp[1].tn_begin) + (int)(tn >= q->grp[2].tn_begin) : 0;
   };
-  auto tile_in_group = [&](int tn, int g) -> int { return GROUPED ? tn - p.grp[g].tn_begin : tn; };
+  auto tile_in_group = [&](int tn, int g) -> int { return GROUPED ? tn - q->grp[g].tn_begin : tn; };
   // Tiles are numbered with the row-tile index fastest.  Each role walks its tiles by adding the
   // stride split into (row tiles, column tiles) once here: a division per tile would sit on the
   // epilogue's and the producer's path.
-  const int step_tn = tile_step / p.tiles_m, step_tm = tile_step - step_tn * p.tiles_m;
-  const int tm0 = tile0 % p.tiles_m, tn0 = tile0 / p.tiles_m;
+  int num_tiles, step_tn, step_tm, tm0, tn0;
+  auto set_record = [&](int li) {
+    q = &L.rec[CHAIN ? li : 0].p;
+    mp = &L.rec[CHAIN ? li : 0].maps;
+    num_tiles = q->tiles_m * q->tiles_n;
+    step_tn = tile_step / q->tiles_m; step_tm = tile_step - step_tn * q->tiles_m;
+    tm0 = tile0 % q->tiles_m; tn0 = tile0 / q->tiles_m;
+  };
+  set_record(0);
+  // chains: position in the launch's tile sequence
+  struct Cur { int li, first, ntiles; const GemmParams* q; const AllMaps* mp; };
+  auto cur_seek = [&](Cur& c, int g) {       // g < L.total_tiles
+    while (g >= c.first + c.ntiles) {
+      c.first += c.ntiles; ++c.li;
+      c.q = &L.rec[CHAIN ? c.li : 0].p; c.mp = &L.rec[CHAIN ? c.li : 0].maps;
+      c.ntiles = c.q->tiles_m * c.q->tiles_n;
+    }
+  };
+  Cur cur{0, 0, num_tiles, q, mp};
+  const int total_tiles = CHAIN ? L.total_tiles : num_tiles;
 
   // producer state (thread 0 only): next k-block to load
   // The producer and the MMA issuer share their scheduler with four epilogue warps that almost
@@ -597,11 +682,11 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   uint32_t ld_dst = stage0, ld_bar = full0;      // stage address and its full barrier
   int ld_x = 0, ld_ya = 0, ld_yb = 0;            // TMA coordinates of the next k-block
   int ld_tm = tm0, ld_tn = tn0;
-  const CUtensorMap* ld_map_a = &maps.g[0].a;
-  const CUtensorMap* ld_map_b = &maps.g[0].b;
+  const CUtensorMap* ld_map_a = &mp->g[0].a;
+  const CUtensorMap* ld_map_b = &mp->g[0].b;
   auto set_tile_coords = [&]() {
     const int g = group_of(ld_tn);
-    if (GROUPED) { ld_map_a = &maps.g[g].a; ld_map_b = &maps.g[g].b; }
+    if (GROUPED) { ld_map_a = &mp->g[g].a; ld_map_b = &mp->g[g].b; }
     ld_ya = ld_tm * rows_per_tile + rank * BM;
     ld_yb = tile_in_group(ld_tn, g) * p.bn + rank * b_rows;
   };
@@ -625,20 +710,21 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
     }
     ld_dst += stage_bytes; ld_bar += 8; ld_x += k_elems;
     if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; ld_dst = stage0; ld_bar = full0; }
-    if (++ld_kb == p.k_blocks) {
+    if (++ld_kb == q->k_blocks) {
       ld_kb = 0; ld_x = 0; ld_tile += tile_step;
       ld_tm += step_tm; ld_tn += step_tn;
-      if (ld_tm >= p.tiles_m) { ld_tm -= p.tiles_m; ++ld_tn; }
+      if (ld_tm >= q->tiles_m) { ld_tm -= q->tiles_m; ++ld_tn; }
       set_tile_coords();
     }
   };
 
   if (threadIdx.x == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.g[0].a) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.g[0].b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&mp->g[0].a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&mp->g[0].b) : "memory");
     const uint32_t full_count = 1 + (p.conv.on ? kGatherWarps * (PAIR ? 2 : 1) : 0);   // the TMA thread, plus one arrival per gather warp
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
+    if (CHAIN) for (int a = 0; a < 4; ++a) mbar_init(done0 + 8 * a, kEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -661,7 +747,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   if (p.stamp && threadIdx.x == 32) atomicMin(p.stamp, (unsigned long long)global_timer());
   if (warp == 0) {
     // the ring is empty: fill it before the block-wide barrier so the first tiles are in flight
-    for (int i = 0; i < p.stages && ld_tile < num_tiles; ++i) issue_load();
+    if (!CHAIN) for (int i = 0; i < p.stages && ld_tile < num_tiles; ++i) issue_load();
   }
   tc_fence_before();
   __syncthreads();
@@ -672,9 +758,50 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
-    while (ld_tile < num_tiles) {
-      if (!mbar_wait_warp(ld_bar + 8 * kMaxStages, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
-      issue_load();
+    if (CHAIN) {
+      int chk_li = -1, chk_tm = -1;
+      for (int g = tile0; g < total_tiles && ok; g += tile_step) {
+        cur_seek(cur, g);
+        const GemmParams* cq = cur.q;
+        const int T = g - cur.first;
+        const int tm = T / cq->tiles_n, tn = T - tm * cq->tiles_n;
+        if (cur.li != chk_li || tm != chk_tm) {      // the rows this tile reads must be complete
+          chk_li = cur.li; chk_tm = tm;
+          bool failed = false;
+          if (elected) {
+            bool waited = false;
+            for (int d = 0; d < kMaxDeps && !failed; ++d) {
+              const int dep = cq->deps[d];
+              if (dep < 0) continue;
+              waited = true;
+              failed = !flag_wait(L.flags + (size_t)dep * L.flag_stride + 2 * tm + rank, (uint32_t)L.rec[dep].p.tiles_n, abort_flag, p.err);
+            }
+            if (waited) asm volatile("fence.proxy.async;" ::: "memory");
+          }
+          if (__any_sync(0xffffffffu, failed)) { ok = false; break; }
+        }
+        const int gi = (int)(tn >= cq->grp[1].tn_begin) + (int)(tn >= cq->grp[2].tn_begin);
+        const CUtensorMap* ma = &cur.mp->g[gi].a;
+        const CUtensorMap* mb = &cur.mp->g[gi].b;
+        const int ya = tm * rows_per_tile + rank * BM;
+        const int yb = (tn - cq->grp[gi].tn_begin) * p.bn + rank * b_rows;
+        int x = 0;
+        for (int kb = 0; kb < cq->k_blocks; ++kb) {
+          if (!mbar_wait_warp(ld_bar + 8 * kMaxStages, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
+          if (elected) {
+            if (rank == 0) mbar_expect_tx(ld_bar, 2 * stage_bytes);
+            tma_load_2d_pair(ld_dst, ma, ld_bar, x, ya);
+            tma_load_2d_pair(ld_dst + BM * kStageKBytes, mb, ld_bar, x, yb);
+          }
+          ld_dst += stage_bytes; ld_bar += 8; x += k_elems;
+          if (++ld_s == p.stages) { ld_s = 0; ld_ph ^= 1; ld_dst = stage0; ld_bar = full0; }
+        }
+      }
+    } else {
+      while (ld_tile < num_tiles) {
+        if (!mbar_wait_warp(ld_bar + 8 * kMaxStages, ld_ph ^ 1, abort_flag, p.err)) { ok = false; break; }
+        issue_load();
+      }
     }
     if (PAIR && ok) {
       // the peer's MMA completions still arrive on this CTA's stage barriers: drain them all
@@ -714,12 +841,13 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
           else tc_mma<BF16>(d_tmem, da, db, p.idesc, acc);
         }
       };
-      for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
+      for (int tile = tile0; tile < total_tiles && ok; tile += tile_step, ++t) {
+        if (CHAIN) { cur_seek(cur, tile); q = cur.q; }
         const int a = t & 1;
         if (!mbar_wait_warp(tempty0 + 8 * a, ((t >> 1) & 1) ^ 1, abort_flag, p.err)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)a * kAccCols;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = 0; kb < q->k_blocks; ++kb) {
           if (!mbar_wait_warp(fb, ph, abort_flag, p.err)) { ok = false; break; }
           tc_fence_after();
           mma4(d_tmem, kb != 0);
@@ -729,6 +857,24 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
           if (++s == p.stages) { s = 0; ph ^= 1; lo = lo0; fb = full0; }
         }
         if (ok && elected) { if (PAIR) tc_commit_pair(tfull0 + 8 * a); else tc_commit(tfull0 + 8 * a); }   // accumulator complete
+      }
+    }
+  } else if (CHAIN && warp >= 2 + kEpiWarps) {
+    // ------------------------------------------------------------------ signal warp (chains)
+    // For each of this CTA's tiles in order: once all epilogue warps have seen their stores of
+    // the tile complete, publish it (release at device scope after the proxy fence that orders
+    // the TMA stores) by adding one to the counter of its record, row tile and CTA rank.
+    if (warp == 2 + kEpiWarps) {
+      int t = 0;
+      for (int g = tile0; g < total_tiles; g += tile_step, ++t) {
+        cur_seek(cur, g);
+        if (!mbar_wait_warp(done0 + 8 * (t & 3), (uint32_t)(t >> 2) & 1u, abort_flag, p.err)) break;
+        if (elected && cur.q->signal) {
+          const int tm = (g - cur.first) / cur.q->tiles_n;
+          asm volatile("fence.proxy.async;" ::: "memory");
+          asm volatile("red.release.gpu.global.add.u32 [%0], 1;"
+                       ::"l"(L.flags + (size_t)cur.li * L.flag_stride + 2 * tm + rank) : "memory");
+        }
       }
     }
   } else if (warp >= 2 + kEpiWarps) {
@@ -817,13 +963,13 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
     // Weight scales of this warp's chunks, one column per lane and chunk.  They are fetched one
     // tile ahead: when the epilogue is the longer phase the accumulator is already waiting at
     // the top of the loop, and a load issued there would put its whole latency on the tile.
-    auto load_scales = [&](int tile, int tile_tn, float (&w)[2]) {
+    auto load_scales = [&](const GemmParams* qq, bool valid, int tile_tn, float (&w)[2]) {
       w[0] = 0.f; w[1] = 0.f;
-      if (BF16 || tile >= num_tiles) return;
-      const int gi = group_of(tile_tn);
-      const GroupDesc& G = p.grp[gi];
+      if (BF16 || !valid) return;
+      const int gi = GROUPED ? (int)(tile_tn >= qq->grp[1].tn_begin) + (int)(tile_tn >= qq->grp[2].tn_begin) : 0;
+      const GroupDesc& G = qq->grp[gi];
       if (!G.need_y) return;
-      const int cb = tile_in_group(tile_tn, gi) * p.bn + c_begin * 32;
+      const int cb = (GROUPED ? tile_tn - G.tn_begin : tile_tn) * p.bn + c_begin * 32;
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int col = cb + j * 32 + lane;
@@ -831,18 +977,51 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
       }
     };
     float sw_next[2];
-    load_scales(tile0, tn0, sw_next);
     int tm = tm0, tn = tn0;
-    for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++t) {
+    if (CHAIN) {
+      if (tile0 < total_tiles) {
+        cur_seek(cur, tile0);
+        load_scales(cur.q, true, (tile0 - cur.first) % cur.q->tiles_n, sw_next);
+      }
+    } else {
+      load_scales(q, tile0 < num_tiles, tn0, sw_next);
+    }
+    for (int tile = tile0; tile < total_tiles && ok; tile += tile_step, ++t) {
+      if (CHAIN) {     // record of this tile, column tile fastest inside it
+        cur_seek(cur, tile); q = cur.q; mp = cur.mp;
+        const int T = tile - cur.first;
+        tm = T / q->tiles_n; tn = T - tm * q->tiles_n;
+      }
       const int a = t & 1;
       const int row0 = tm * rows_per_tile + rank * BM + quad * 32;
       const int g = group_of(tn);
-      const GroupDesc& G = p.grp[g];
+      const GroupDesc& G = q->grp[g];
       const int col_base = tile_in_group(tn, g) * p.bn + c_begin * 32;
       const float cs[2] = {__fmul_rn(G.scale_x, sw_next[0]), __fmul_rn(G.scale_x, sw_next[1])};
       int tm_next = tm + step_tm, tn_next = tn + step_tn;
-      if (tm_next >= p.tiles_m) { tm_next -= p.tiles_m; ++tn_next; }
-      load_scales(tile + tile_step, tn_next, sw_next);
+      if (CHAIN) {
+        const int nt = tile + tile_step;
+        Cur c2 = cur;
+        if (nt < total_tiles) cur_seek(c2, nt);
+        load_scales(c2.q, nt < total_tiles, nt < total_tiles ? (nt - c2.first) % c2.q->tiles_n : 0, sw_next);
+      } else {
+        if (tm_next >= q->tiles_m) { tm_next -= q->tiles_m; ++tn_next; }
+        load_scales(q, tile + tile_step < num_tiles, tn_next, sw_next);
+      }
+      // Chains: the previous tile is reported once its stores have completed.  When this tile's
+      // accumulator is already there the check is left to the body (just before its first store,
+      // when the old stores have long landed); when it is not, this tile may itself be waiting for
+      // rows other CTAs produce, and they for the report, so the report goes out now.
+      uint32_t done_bar = (CHAIN && t > 0) ? done0 + 8 * ((t - 1) & 3) : 0u;
+      const bool fast_inside = G.mode != EPI_GENERAL && !(row0 >= q->m || col_base >= G.n);
+      if (done_bar && !(fast_inside && __all_sync(0xffffffffu, mbar_try_wait(tfull0 + 8 * a, (t >> 1) & 1)))) {
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+          mbar_arrive(done_bar);
+        }
+        __syncwarp();
+        done_bar = 0;
+      }
       if (!mbar_wait(tfull0 + 8 * a, (t >> 1) & 1, abort_flag, p.err)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a * kAccCols + c_begin * 32);
@@ -851,7 +1030,7 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
       const uint32_t tempty_bar = tempty0 + 8 * a;
       if (G.mode != EPI_GENERAL) {
         // fast bodies: 256-column tiles, so this warp owns 64 columns starting at col_base
-        if (row0 >= p.m || col_base >= G.n) {
+        if (!fast_inside) {
           __syncwarp();
           if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
         } else {
@@ -861,9 +1040,9 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
             __syncwarp();
           }
           if (G.mode == EPI_CODES1)
-            epilogue_tile_fast<BF16, PAIR, true>(G, &maps.g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar);
+            epilogue_tile_fast<BF16, PAIR, true>(G, &mp->g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
           else
-            epilogue_tile_fast<BF16, PAIR, false>(G, &maps.g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar);
+            epilogue_tile_fast<BF16, PAIR, false>(G, &mp->g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
         }
         prev_fast = true;
       } else {
@@ -884,14 +1063,20 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
             if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
           }
           const float csl = c ? cs[1] : cs[0];
-          epilogue_chunk<BF16>(G, maps.g[g].om, p.m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
+          epilogue_chunk<BF16>(G, mp->g[g].om, q->m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
         }
         if (nch == 0) {
           __syncwarp();
           if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
         }
       }
-      tm = tm_next; tn = tn_next;
+      if (!CHAIN) { tm = tm_next; tn = tn_next; }
+    }
+    if (CHAIN && t > 0 && ok) {       // the last tile: report it as soon as its stores have completed
+      if (lane == 0) {
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        mbar_arrive(done0 + 8 * ((t - 1) & 3));
+      }
     }
     // all TMA stores of this warp must have completed before the CTA's shared memory goes away
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -909,6 +1094,26 @@ gemm_kernel(const __grid_constant__ AllMaps maps, const __grid_constant__ GemmPa
 }
 
 // ---------------------------------------------------------------------------- host side
+
+// Host state of the chain being collected (one per context).
+struct Span { const uint8_t* lo; const uint8_t* hi; };      // byte range [lo, hi) of a matrix
+struct ChainRecInfo { Span in[2 * kMaxGroups]; int n_in; Span out[kNumOuts * kMaxGroups]; int n_out; };
+constexpr size_t kFlagRingBytes = 8u << 20;
+constexpr int kChainMaxTilesM = 2048;
+struct ChainState {
+  LaunchArgs<kChainMax> args;     // args.n records collected so far
+  ChainRecInfo info[kChainMax];
+  double ops = 0.0;
+  unsigned* ring = nullptr;       // device counters, handed out front to back and cleared when used up
+  size_t ring_used = 0;           // bytes
+  bool open = false;              // a forward pass is running: eligible launches may be deferred
+  bool bf16 = false;
+  int grid = 0;
+  int64_t m = 0;
+  size_t smem = 0;
+  cudaStream_t st = nullptr;
+  ChainState() { memset(&args, 0, sizeof(args)); }
+};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1025,14 +1230,101 @@ int gemm_init(Ctx* ctx) {
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
   cudaError_t e = cudaSuccess;
-  const void* kernels[8] = {
-      (const void*)gemm_kernel<false, false, false>, (const void*)gemm_kernel<false, false, true>,
-      (const void*)gemm_kernel<false, true, false>,  (const void*)gemm_kernel<false, true, true>,
-      (const void*)gemm_kernel<true, false, false>,  (const void*)gemm_kernel<true, false, true>,
-      (const void*)gemm_kernel<true, true, false>,   (const void*)gemm_kernel<true, true, true>};
-  for (int i = 0; i < 8 && e == cudaSuccess; ++i)
+  const void* kernels[10] = {
+      (const void*)gemm_kernel<false, false, false, false>, (const void*)gemm_kernel<false, false, true, false>,
+      (const void*)gemm_kernel<false, true, false, false>,  (const void*)gemm_kernel<false, true, true, false>,
+      (const void*)gemm_kernel<true, false, false, false>,  (const void*)gemm_kernel<true, false, true, false>,
+      (const void*)gemm_kernel<true, true, false, false>,   (const void*)gemm_kernel<true, true, true, false>,
+      (const void*)gemm_kernel<false, true, true, true>,    (const void*)gemm_kernel<true, true, true, true>};
+  for (int i = 0; i < 10 && e == cudaSuccess; ++i)
     e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
-  return check_cuda(ctx, e, "gemm smem attribute");
+  if (e != cudaSuccess) return check_cuda(ctx, e, "gemm smem attribute");
+  ChainState* cs = new (std::nothrow) ChainState();
+  if (!cs) return set_error(ctx, QCFG_ENOMEM, "gemm: host allocation failed");
+  e = cudaMalloc(&cs->ring, kFlagRingBytes);
+  if (e == cudaSuccess) e = cudaMemset(cs->ring, 0, kFlagRingBytes);
+  if (e != cudaSuccess) { delete cs; return check_cuda(ctx, e, "gemm chain counters"); }
+  chain_slot(ctx) = cs;
+  return QCFG_OK;
+}
+
+void gemm_destroy(Ctx* ctx) {
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  if (!cs) return;
+  if (cs->ring) cudaFree(cs->ring);
+  delete cs;
+  chain_slot(ctx) = nullptr;
+}
+
+// ----- chains: consecutive GEMM launches of a forward pass folded into one cooperative launch
+
+void gemm_chain_open(Ctx* ctx) {
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  if (cs && ctx_chain_enabled(ctx)) cs->open = true;
+}
+
+int gemm_chain_flush(Ctx* ctx) {
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  if (!cs || cs->args.n == 0) return QCFG_OK;
+  const int n = cs->args.n;
+  cs->args.n = 0;
+  LaunchArgs<kChainMax>& A = cs->args;
+  // counters: two per row tile and record, from a region nobody has used since it was cleared
+  const int stride = 2 * A.rec[0].p.tiles_m;
+  const size_t need = (size_t)n * stride * sizeof(unsigned);
+  if (cs->ring_used + need > kFlagRingBytes) {
+    // used up (once in a few thousand launches): wait for every launch that may still read it
+    cudaError_t me = cudaDeviceSynchronize();
+    if (me == cudaSuccess) me = cudaMemsetAsync(cs->ring, 0, kFlagRingBytes, cs->st);
+    if (me != cudaSuccess) return check_cuda(ctx, me, "gemm chain counters");
+    cs->ring_used = 0;
+  }
+  A.flags = cs->ring + cs->ring_used / sizeof(unsigned);
+  cs->ring_used += need;
+  A.flag_stride = stride;
+  A.n = n;
+  int total = 0;
+  for (int i = 0; i < n; ++i) total += A.rec[i].p.tiles_m * A.rec[i].p.tiles_n;
+  A.total_tiles = total;
+  A.rec[0].p.stamp = prof_stamp(ctx, cs->bf16 ? 1 : 0, cs->ops);
+  cs->ops = 0.0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)cs->grid);
+  cfg.blockDim = dim3(kGemmThreads + 32);      // one more warp: it publishes the finished tiles
+  cfg.dynamicSmemBytes = cs->smem;
+  cfg.stream = cs->st;
+  cudaLaunchAttribute attr[3];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  attr[2].id = cudaLaunchAttributeCooperative;      // CTAs wait for tiles of other CTAs
+  attr[2].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 3;
+  const cudaError_t le = cs->bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, true, true, true>, A)
+                                  : cudaLaunchKernelEx(&cfg, gemm_kernel<false, true, true, true>, A);
+  A.n = 0;
+  if (le != cudaSuccess) return check_cuda(ctx, le, "gemm chain launch");
+  count_launch(ctx);
+  return check_cuda(ctx, cudaGetLastError(), "gemm chain launch");
+}
+
+int gemm_chain_close(Ctx* ctx) {
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  if (!cs) return QCFG_OK;
+  cs->open = false;
+  return gemm_chain_flush(ctx);
+}
+
+// After a device-side wait gave up, counters of unfinished launches may be left behind.
+int gemm_chain_reset(Ctx* ctx) {
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  if (!cs) return QCFG_OK;
+  cs->args.n = 0;
+  cs->ops = 0.0;
+  cs->ring_used = 0;
+  return check_cuda(ctx, cudaMemset(cs->ring, 0, kFlagRingBytes), "gemm chain counters reset");
 }
 
 // Tile width a GEMM of n columns gets.
@@ -1133,7 +1425,11 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
     if (cv.OH < 1 || cv.OW < 1 || g0.m % ((int64_t)cv.OH * cv.OW))
       return set_error(ctx, QCFG_ESHAPE, "gemm: convolution rows are not a whole number of images");
   }
-  p.epi_bytes = wide ? 4096 : 2048;
+  // Launches that may join a chain all take the larger staging size, so any sequence of them
+  // shares one shared-memory layout.
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  const bool chainable = cs && cs->open && pair && !conv && bn == 256 && prof_mode(ctx) != 1 && p.tiles_m <= kChainMaxTilesM;
+  p.epi_bytes = (wide || chainable) ? 4096 : 2048;
   int stages = (kSmemMax - kSmemHeader - kCsBytes - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages <= kGatherDepth) return set_error(ctx, QCFG_ESHAPE, "gemm: too few pipeline stages");
@@ -1153,16 +1449,80 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
       q.attrs = qa; q.numAttrs = 1;
       int n = 0;
-      cudaError_t oe = g0.is_bf16 ? cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true, true, false>, &q)
-                                  : cudaOccupancyMaxActiveClusters(&n, gemm_kernel<false, true, false>, &q);
+      cudaError_t oe = g0.is_bf16 ? cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true, true, true, true>, &q)
+                                  : cudaOccupancyMaxActiveClusters(&n, gemm_kernel<false, true, true, true>, &q);
       if (oe != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = grid / 2; }
       if (n > grid / 2) n = grid / 2;
       *cached = n;
     }
     grid = 2 * (*cached);
-    if (grid > 2 * num_tiles) grid = 2 * num_tiles;
+    if (grid > 2 * num_tiles && !chainable) grid = 2 * num_tiles;
   } else if (grid > num_tiles) grid = num_tiles;
   const size_t smem = (size_t)kSmemHeader + kCsBytes + 1024 + (size_t)kEpiWarps * p.epi_bytes + (size_t)stages * stage_bytes;
+  if (cs && cs->args.n > 0 &&
+      (!chainable || cs->args.n == kChainMax || cs->st != st || cs->bf16 != (g0.is_bf16 != 0) || cs->grid != grid ||
+       cs->smem != smem || cs->m != g0.m)) {
+    const int rc = gemm_chain_flush(ctx);
+    if (rc != QCFG_OK) return rc;
+  }
+  if (chainable) {
+    // What the record reads and writes, as byte ranges.  Reading rows an earlier record of the
+    // chain writes is a dependency the kernel waits for; any other overlap ends the chain first.
+    ChainRecInfo info{};
+    bool b_clash = false;
+    auto overlap = [](const Span& x, const Span& y) { return x.lo < y.hi && y.lo < x.hi; };
+    auto span_of = [&](const void* ptr, int64_t ld, int64_t cols, int esz_) {
+      const uint8_t* lo = static_cast<const uint8_t*>(ptr);
+      return Span{lo, lo + ((g0.m - 1) * ld + cols) * esz_};
+    };
+    for (int i = 0; i < count; ++i) {
+      const GemmArgs& g = gs[i];
+      info.in[info.n_in++] = span_of(g.a, g.lda, g.k, esz);
+      if (g.residual) info.in[info.n_in++] = span_of(g.residual, g.ldr, g.n, 4);
+      for (int j = 0; j < kNumOuts; ++j) {
+        const OutDesc& o = p.grp[i].outs[j];
+        if (o.kind) info.out[info.n_out++] = span_of(o.ptr, o.ld, g.n, o.kind == 1 ? 1 : o.kind == 2 ? 2 : 4);
+      }
+      // weights and their scales are never chain outputs in a forward pass; if they were, run apart
+      const uint8_t* blo = static_cast<const uint8_t*>(g.b);
+      const Span bs{blo, blo + ((g.n - 1) * g.ldb + g.k) * esz};
+      for (int r = 0; r < cs->args.n; ++r)
+        for (int o = 0; o < cs->info[r].n_out; ++o) b_clash = b_clash || overlap(bs, cs->info[r].out[o]);
+    }
+    int deps[kMaxDeps], n_deps = 0;
+    bool clash = b_clash;
+    for (int r = 0; r < cs->args.n && !clash; ++r) {
+      const ChainRecInfo& E = cs->info[r];
+      for (int o = 0; o < info.n_out && !clash; ++o) {
+        for (int x = 0; x < E.n_in; ++x) clash = clash || overlap(info.out[o], E.in[x]);
+        for (int x = 0; x < E.n_out; ++x) clash = clash || overlap(info.out[o], E.out[x]);
+      }
+      bool reads = false;
+      for (int x = 0; x < info.n_in; ++x)
+        for (int o = 0; o < E.n_out; ++o) reads = reads || overlap(info.in[x], E.out[o]);
+      if (reads) {
+        if (n_deps == kMaxDeps) clash = true;
+        else deps[n_deps++] = r;
+      }
+    }
+    if (clash) {
+      const int rc = gemm_chain_flush(ctx);
+      if (rc != QCFG_OK) return rc;
+      n_deps = 0;
+    }
+    for (int d = 0; d < kMaxDeps; ++d) p.deps[d] = d < n_deps ? deps[d] : -1;
+    for (int d = 0; d < n_deps; ++d) cs->args.rec[deps[d]].p.signal = 1;
+    p.signal = 0;
+    p.stamp = nullptr;
+    const int slot = cs->args.n++;
+    cs->args.rec[slot].maps = maps;
+    cs->args.rec[slot].p = p;
+    cs->info[slot] = info;
+    cs->ops += ops;
+    cs->st = st; cs->bf16 = g0.is_bf16 != 0; cs->grid = grid; cs->smem = smem; cs->m = g0.m;
+    return QCFG_OK;
+  }
+  for (int d = 0; d < kMaxDeps; ++d) p.deps[d] = -1;
   // Programmatic dependent launch: the kernel's prologue (barrier set-up, TMEM allocation) may
   // start while the previous kernel in the stream drains; it waits (griddepcontrol.wait) before
   // touching global memory.
@@ -1178,14 +1538,19 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
   attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 2 : 1;
-  using Kern = void (*)(const AllMaps, const GemmParams);
+  using Kern = void (*)(const LaunchArgs<1>);
   static const Kern kernels[8] = {
-      gemm_kernel<false, false, false>, gemm_kernel<false, false, true>, gemm_kernel<false, true, false>, gemm_kernel<false, true, true>,
-      gemm_kernel<true, false, false>,  gemm_kernel<true, false, true>,  gemm_kernel<true, true, false>,  gemm_kernel<true, true, true>};
+      gemm_kernel<false, false, false, false>, gemm_kernel<false, false, true, false>, gemm_kernel<false, true, false, false>,
+      gemm_kernel<false, true, true, false>,   gemm_kernel<true, false, false, false>,  gemm_kernel<true, false, true, false>,
+      gemm_kernel<true, true, false, false>,   gemm_kernel<true, true, true, false>};
   const Kern kern = kernels[(g0.is_bf16 ? 4 : 0) + (pair ? 2 : 0) + (count > 1 ? 1 : 0)];
   p.stamp = prof_stamp(ctx, g0.is_bf16 ? 1 : 0, ops);
+  static thread_local LaunchArgs<1> one;
+  one.rec[0].maps = maps;
+  one.rec[0].p = p;
+  one.n = 1; one.total_tiles = num_tiles; one.flag_stride = 0; one.flags = nullptr;
   prof_begin(ctx, g0.is_bf16 ? 1 : 0, st);
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, maps, p);
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, kern, one);
   prof_end(ctx, g0.is_bf16 ? 1 : 0, ops, st);
   if (le != cudaSuccess) return check_cuda(ctx, le, "gemm launch");
   count_launch(ctx);

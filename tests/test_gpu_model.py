@@ -281,3 +281,39 @@ def test_implicit_and_materialised_convolutions_agree_bitwise(ctx, fuse):
         ctx.set_implicit_conv(True)
         ctx.set_fusion(True)
         model.close()
+
+
+@pytest.mark.parametrize("m", [1664, 700])
+def test_chained_and_separate_launches_agree_bitwise(ctx, m):
+    """A forward pass whose GEMMs go to the device as chains (one cooperative launch for up to seven
+    consecutive layers, tiles started by per-row-tile counters) gives the same bits as one launch
+    per GEMM: all-int8, a mix with 4-bit and 16-bit layers (both operand types chain), every
+    output requested (general epilogue) and only the last one (fast epilogue bodies), whole and
+    ragged last row tiles.  The launch counter shows that the chains were in fact used."""
+    w = wl.bert_stack(11, m, 256, 1024, 3, bit_choices=None)
+    model, x = build(ctx, w)
+    n = len(w.layers)
+    mixed = [16 if i % 5 == 4 else (4 if i % 3 == 0 else 8) for i in range(n)]
+    last = torch.empty((m, w.layers[-1].n_out), device="cuda")
+    try:
+        for bits in ([8] * n, mixed, [16] * n):
+            outs, lasts, launches = {}, {}, {}
+            for chained in (True, False):
+                ctx.set_gemm_chains(chained)
+                ys = run_eval(ctx, model, w, x, bits)
+                outs[chained] = [host(y) for y in ys]
+                last.fill_(float("nan"))
+                n0 = ctx.launch_count()
+                model.eval_config(bits, x, m, [None] * (n - 1) + [last])
+                ctx.check_sync()
+                launches[chained] = ctx.launch_count() - n0
+                lasts[chained] = host(last).copy()
+            for l in range(n):
+                np.testing.assert_array_equal(outs[True][l].view(np.uint32), outs[False][l].view(np.uint32),
+                                              err_msg=f"layer {l} ({w.layers[l].name}) bits {bits[l]}")
+            np.testing.assert_array_equal(lasts[True].view(np.uint32), lasts[False].view(np.uint32))
+            assert np.all(np.isfinite(lasts[True]))
+            assert launches[True] < launches[False], launches
+    finally:
+        ctx.set_gemm_chains(True)
+        model.close()
