@@ -73,6 +73,9 @@ struct GroupDesc {
   int32_t act;
   int32_t need_y;             // anything besides raw accumulators to produce
   int32_t mode;               // EPI_*: which epilogue body serves this group
+  // chains number a record's tiles group by group (column tile fastest inside a group):
+  int32_t gtiles_n, tile_first;   // column tiles of this group; record-local index of its first tile (unused: INT32_MAX)
+  int32_t signal;             // a later record of the launch reads this group's output rows
   float scale_x;
   const float* scale_w;
   const float* residual; int64_t ldr;
@@ -98,7 +101,7 @@ struct GemmParams {
   // chains: records of the same launch whose output rows this record reads (-1: none), and
   // whether a later record of the launch reads this one's
   int32_t deps[kMaxDeps];
-  int32_t signal;
+  int32_t need;               // finished tiles per row tile and CTA rank that make this record's rows complete for its readers
 };
 // What one launch gets: one record, or a chain of them (see the kernel).
 constexpr int kChainMax = 7;
@@ -166,6 +169,26 @@ __device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, v
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (v >= need) return true;
     if ((it & 63u) == 0) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
+        atomicOr(err, ERR_TIMEOUT);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+// Chains: waits until the CTA's dependency warp has cleared `need` tiles (a counter in shared memory).
+__device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volatile int* abort_flag, unsigned* err) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    if (v >= need) return true;
+    if ((it & 1023u) == 0) {
       if (*abort_flag) return false;
       const uint64_t now = global_timer();
       if (t0 == 0) t0 = now;
@@ -446,7 +469,7 @@ __device__ __forceinline__ float2 code_words2(float2 y, float2 inv2, float qmax)
 // rows (128B swizzle), one TMA store per block; the single staging slot is reused once the
 // previous store has read it.
 // done_bar (chains, else 0): barrier to arrive on once the stores this warp issued for its previous
-// tile have completed; that is checked just before this tile's first store, most of an epilogue
+// tile have completed; that is checked after this tile's first piece, a quarter of an epilogue
 // after they were issued.
 template <bool BF16, bool PAIR, bool CODES>
 __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUtensorMap* fmap, uint32_t tbase,
@@ -488,6 +511,10 @@ __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUt
       __syncwarp();
     }
     piece(va, 2 * h);
+    if (h == 0 && done_bar && lane == 0) {    // a quarter of a tile after the previous tile's last store
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      mbar_arrive(done_bar);
+    }
     tmem_ld_wait();
     if (h == 0) {
       tmem_ld16_issue(tbase + 32, va);
@@ -500,25 +527,13 @@ __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUt
     if (!CODES) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) {
-        if (h == 0 && done_bar) {
-          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-          mbar_arrive(done_bar);
-        }
-        if (col0 + 32 * h < G.n) tma_store_2d(fmap, stage, col0 + 32 * h, row0);
-      }
+      if (lane == 0 && col0 + 32 * h < G.n) tma_store_2d(fmap, stage, col0 + 32 * h, row0);
     }
   }
   if (CODES) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    if (lane == 0) {
-      if (done_bar) {
-        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        mbar_arrive(done_bar);
-      }
-      tma_store_2d(fmap, stage, col0, row0);
-    }
+    if (lane == 0) tma_store_2d(fmap, stage, col0, row0);
   }
 }
 
@@ -601,7 +616,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
 
 // One launch runs one GEMM record or, in the CHAIN flavour, up to kChainMax records one after the
 // other: consecutive layers of a model, each reading what an earlier one wrote.  The tiles of all
-// records form one sequence (record after record, column tile fastest inside a record) that the
+// records form one sequence (record after record, group after group, column tile fastest) that the
 // CTA pairs deal out round-robin, so a pair that runs out of tiles of one record goes on with the
 // next: no pipeline fill and drain, no idle last round and no kernel boundary between layers.
 // A tile may start when the row tiles it reads are complete: every finished tile adds one to a
@@ -622,6 +637,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);           // full[8] empty[8] tfull[2] tempty[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
+  const uint32_t cleared_addr = smem_u32(smem + 264);            // chains: tiles of this CTA whose inputs are complete
   float* cs_all = reinterpret_cast<float*>(smem + kSmemHeader);  // kEpiWarps x 64 rescale factors
   uint8_t* epi_stage = smem + kSmemHeader + kCsBytes;            // kEpiWarps x epi_bytes, 1024-aligned
   uint8_t* stage_base = epi_stage + kEpiWarps * p.epi_bytes;
@@ -668,6 +684,14 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
     }
   };
   Cur cur{0, 0, num_tiles, q, mp};
+  // record-local tile index -> group, row tile, column tile (column tiles numbered over all groups)
+  auto locate = [&](const GemmParams* qq, int T, int& gi, int& tm, int& tn) {
+    gi = (int)(T >= qq->grp[1].tile_first) + (int)(T >= qq->grp[2].tile_first);
+    const GroupDesc& G = qq->grp[gi];
+    const int Tl = T - G.tile_first;
+    tm = Tl / G.gtiles_n;
+    tn = G.tn_begin + (Tl - tm * G.gtiles_n);
+  };
   const int total_tiles = CHAIN ? L.total_tiles : num_tiles;
 
   // producer state (thread 0 only): next k-block to load
@@ -726,6 +750,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
     if (CHAIN) for (int a = 0; a < 4; ++a) mbar_init(done0 + 8 * a, kEpiWarps);
     *abort_flag = 0;
+    *reinterpret_cast<volatile uint32_t*>(smem + 264) = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -759,28 +784,15 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
     if (CHAIN) {
-      int chk_li = -1, chk_tm = -1;
+      // The dependency warp clears tiles ahead of time (see there); here only a counter in shared
+      // memory is read, so no device-scope fence sits between two tiles' loads.
+      uint32_t t_ld = 0;
       for (int g = tile0; g < total_tiles && ok; g += tile_step) {
         cur_seek(cur, g);
         const GemmParams* cq = cur.q;
-        const int T = g - cur.first;
-        const int tm = T / cq->tiles_n, tn = T - tm * cq->tiles_n;
-        if (cur.li != chk_li || tm != chk_tm) {      // the rows this tile reads must be complete
-          chk_li = cur.li; chk_tm = tm;
-          bool failed = false;
-          if (elected) {
-            bool waited = false;
-            for (int d = 0; d < kMaxDeps && !failed; ++d) {
-              const int dep = cq->deps[d];
-              if (dep < 0) continue;
-              waited = true;
-              failed = !flag_wait(L.flags + (size_t)dep * L.flag_stride + 2 * tm + rank, (uint32_t)L.rec[dep].p.tiles_n, abort_flag, p.err);
-            }
-            if (waited) asm volatile("fence.proxy.async;" ::: "memory");
-          }
-          if (__any_sync(0xffffffffu, failed)) { ok = false; break; }
-        }
-        const int gi = (int)(tn >= cq->grp[1].tn_begin) + (int)(tn >= cq->grp[2].tn_begin);
+        int gi, tm, tn;
+        locate(cq, g - cur.first, gi, tm, tn);
+        if (!cleared_wait(cleared_addr, ++t_ld, abort_flag, p.err)) { ok = false; break; }
         const CUtensorMap* ma = &cur.mp->g[gi].a;
         const CUtensorMap* mb = &cur.mp->g[gi].b;
         const int ya = tm * rows_per_tile + rank * BM;
@@ -862,18 +874,44 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
   } else if (CHAIN && warp >= 2 + kEpiWarps) {
     // ------------------------------------------------------------------ signal warp (chains)
     // For each of this CTA's tiles in order: once all epilogue warps have seen their stores of
-    // the tile complete, publish it (release at device scope after the proxy fence that orders
-    // the TMA stores) by adding one to the counter of its record, row tile and CTA rank.
+    // the tile complete (the bulk-group wait makes the TMA writes visible to the waiting thread,
+    // whose barrier arrival this warp has acquired), publish it with a release at device scope:
+    // one is added to the counter of its record, row tile and CTA rank.
     if (warp == 2 + kEpiWarps) {
       int t = 0;
       for (int g = tile0; g < total_tiles; g += tile_step, ++t) {
         cur_seek(cur, g);
         if (!mbar_wait_warp(done0 + 8 * (t & 3), (uint32_t)(t >> 2) & 1u, abort_flag, p.err)) break;
-        if (elected && cur.q->signal) {
-          const int tm = (g - cur.first) / cur.q->tiles_n;
-          asm volatile("fence.proxy.async;" ::: "memory");
+        int gi, tm, tn;
+        locate(cur.q, g - cur.first, gi, tm, tn);
+        if (elected && cur.q->grp[gi].signal) {
           asm volatile("red.release.gpu.global.add.u32 [%0], 1;"
                        ::"l"(L.flags + (size_t)cur.li * L.flag_stride + 2 * tm + rank) : "memory");
+        }
+      }
+    } else if (warp == 3 + kEpiWarps) {
+      // ---------------------------------------------------------------- dependency warp (chains)
+      // Walks this CTA's tiles ahead of the producer.  For each, lane d waits (acquire at device
+      // scope, bounded) until the counter of dependency d says the rows the tile reads are
+      // complete; then one lane orders the asynchronous proxy after that and publishes the tile
+      // count in shared memory, which is all the producer looks at.  The two device-scope fences
+      // cost about a microsecond each under load, and here they delay nobody.
+      uint32_t t_clear = 0;
+      for (int g = tile0; g < total_tiles; g += tile_step) {
+        cur_seek(cur, g);
+        int gi, tm, tn;
+        locate(cur.q, g - cur.first, gi, tm, tn);
+        const int dep = lane < kMaxDeps ? cur.q->deps[lane] : -1;
+        bool failed = false;
+        if (dep >= 0)
+          failed = !flag_wait(L.flags + (size_t)dep * L.flag_stride + 2 * tm + rank, (uint32_t)L.rec[dep].p.need, abort_flag, p.err);
+        const bool had = __any_sync(0xffffffffu, dep >= 0);
+        if (__any_sync(0xffffffffu, failed)) break;
+        ++t_clear;
+        __syncwarp();
+        if (elected) {
+          if (had) asm volatile("fence.proxy.async;" ::: "memory");
+          asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(cleared_addr), "r"(t_clear) : "memory");
         }
       }
     }
@@ -981,7 +1019,9 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
     if (CHAIN) {
       if (tile0 < total_tiles) {
         cur_seek(cur, tile0);
-        load_scales(cur.q, true, (tile0 - cur.first) % cur.q->tiles_n, sw_next);
+        int gi0, tm_0, tn_0;
+        locate(cur.q, tile0 - cur.first, gi0, tm_0, tn_0);
+        load_scales(cur.q, true, tn_0, sw_next);
       }
     } else {
       load_scales(q, tile0 < num_tiles, tn0, sw_next);
@@ -989,8 +1029,8 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
     for (int tile = tile0; tile < total_tiles && ok; tile += tile_step, ++t) {
       if (CHAIN) {     // record of this tile, column tile fastest inside it
         cur_seek(cur, tile); q = cur.q; mp = cur.mp;
-        const int T = tile - cur.first;
-        tm = T / q->tiles_n; tn = T - tm * q->tiles_n;
+        int gi_;
+        locate(q, tile - cur.first, gi_, tm, tn);
       }
       const int a = t & 1;
       const int row0 = tm * rows_per_tile + rank * BM + quad * 32;
@@ -1003,14 +1043,16 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
         const int nt = tile + tile_step;
         Cur c2 = cur;
         if (nt < total_tiles) cur_seek(c2, nt);
-        load_scales(c2.q, nt < total_tiles, nt < total_tiles ? (nt - c2.first) % c2.q->tiles_n : 0, sw_next);
+        int gi2 = 0, tm2 = 0, tn2 = 0;
+        if (nt < total_tiles) locate(c2.q, nt - c2.first, gi2, tm2, tn2);
+        load_scales(c2.q, nt < total_tiles, tn2, sw_next);
       } else {
         if (tm_next >= q->tiles_m) { tm_next -= q->tiles_m; ++tn_next; }
         load_scales(q, tile + tile_step < num_tiles, tn_next, sw_next);
       }
       // Chains: the previous tile is reported once its stores have completed.  When this tile's
-      // accumulator is already there the check is left to the body (just before its first store,
-      // when the old stores have long landed); when it is not, this tile may itself be waiting for
+      // accumulator is already there the check is left to the body (after its first piece, when
+      // the old stores have landed); when it is not, this tile may itself be waiting for
       // rows other CTAs produce, and they for the report, so the report goes out now.
       uint32_t done_bar = (CHAIN && t > 0) ? done0 + 8 * ((t - 1) & 3) : 0u;
       const bool fast_inside = G.mode != EPI_GENERAL && !(row0 >= q->m || col_base >= G.n);
@@ -1097,7 +1139,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
 
 // Host state of the chain being collected (one per context).
 struct Span { const uint8_t* lo; const uint8_t* hi; };      // byte range [lo, hi) of a matrix
-struct ChainRecInfo { Span in[2 * kMaxGroups]; int n_in; Span out[kNumOuts * kMaxGroups]; int n_out; };
+struct ChainRecInfo { Span in[2 * kMaxGroups]; int n_in; Span out[kNumOuts * kMaxGroups]; int out_grp[kNumOuts * kMaxGroups]; int n_out; };
 constexpr size_t kFlagRingBytes = 8u << 20;
 constexpr int kChainMaxTilesM = 2048;
 struct ChainState {
@@ -1284,13 +1326,19 @@ int gemm_chain_flush(Ctx* ctx) {
   A.flag_stride = stride;
   A.n = n;
   int total = 0;
-  for (int i = 0; i < n; ++i) total += A.rec[i].p.tiles_m * A.rec[i].p.tiles_n;
+  for (int i = 0; i < n; ++i) {
+    GemmParams& rp = A.rec[i].p;
+    total += rp.tiles_m * rp.tiles_n;
+    rp.need = 0;
+    for (int gi = 0; gi < kMaxGroups; ++gi)
+      if (rp.grp[gi].tn_begin != 0x7fffffff && rp.grp[gi].signal) rp.need += rp.grp[gi].gtiles_n;
+  }
   A.total_tiles = total;
   A.rec[0].p.stamp = prof_stamp(ctx, cs->bf16 ? 1 : 0, cs->ops);
   cs->ops = 0.0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)cs->grid);
-  cfg.blockDim = dim3(kGemmThreads + 32);      // one more warp: it publishes the finished tiles
+  cfg.blockDim = dim3(kGemmThreads + 64);      // two more warps: one publishes finished tiles, one clears tiles whose inputs are complete
   cfg.dynamicSmemBytes = cs->smem;
   cfg.stream = cs->st;
   cudaLaunchAttribute attr[3];
@@ -1335,8 +1383,32 @@ bool gemm_groupable(const GemmArgs& a, const GemmArgs& b) {
   return a.m == b.m && a.k == b.k && a.is_bf16 == b.is_bf16 && tile_n_of(a.n) == tile_n_of(b.n);
 }
 
-int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) {
+int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t st) {
   if (count < 1 || count > kMaxGroups) return set_error(ctx, QCFG_EINVAL, "gemm: %d groups", count);
+  // While launches are being chained a record's tiles run group after group.  Groups that write
+  // operand codes for later layers go in the middle: the groups before them give the previous
+  // record time to complete the rows they read, the groups after them give their own rows time to
+  // complete before the next record asks for them.
+  GemmArgs ordered[kMaxGroups];
+  {
+    ChainState* st_ = static_cast<ChainState*>(chain_slot(ctx));
+    if (st_ && st_->open && count > 1) {
+      int feed[kMaxGroups], n_feed = 0, rest[kMaxGroups], n_rest = 0;
+      for (int i = 0; i < count; ++i) {
+        bool feeds = false;
+        for (int s = 0; s < kMaxSlots; ++s) feeds = feeds || gs_in[i].slots[s].kind != 0;
+        if (feeds) feed[n_feed++] = i; else rest[n_rest++] = i;
+      }
+      int k = 0;
+      const int before = (n_rest + 1) / 2;
+      for (int i = 0; i < before; ++i) ordered[k++] = gs_in[rest[i]];
+      for (int i = 0; i < n_feed; ++i) ordered[k++] = gs_in[feed[i]];
+      for (int i = before; i < n_rest; ++i) ordered[k++] = gs_in[rest[i]];
+    } else {
+      for (int i = 0; i < count; ++i) ordered[i] = gs_in[i];
+    }
+  }
+  const GemmArgs* gs = ordered;
   const GemmArgs& g0 = gs[0];
   const int esz = g0.is_bf16 ? 2 : 1;
   const int bn = tile_n_of(g0.n);
@@ -1377,12 +1449,14 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
   bool wide = false;
   int32_t tn_total = 0;
   double ops = 0.0;
-  for (int i = 0; i < kMaxGroups; ++i) p.grp[i].tn_begin = 0x7fffffff;
+  for (int i = 0; i < kMaxGroups; ++i) { p.grp[i].tn_begin = 0x7fffffff; p.grp[i].tile_first = 0x7fffffff; p.grp[i].gtiles_n = 1; }
   for (int i = 0; i < count; ++i) {
     const GemmArgs& g = gs[i];
     GroupDesc& G = p.grp[i];
     G.n = (int32_t)g.n;
     G.tn_begin = tn_total;
+    G.gtiles_n = (int32_t)((g.n + bn - 1) / bn);
+    G.tile_first = p.tiles_m * tn_total;
     tn_total += (int32_t)((g.n + bn - 1) / bn);
     G.scale_x = g.scale_x; G.scale_w = g.scale_w; G.act = g.act;
     G.residual = g.residual; G.ldr = g.ldr;
@@ -1481,7 +1555,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       if (g.residual) info.in[info.n_in++] = span_of(g.residual, g.ldr, g.n, 4);
       for (int j = 0; j < kNumOuts; ++j) {
         const OutDesc& o = p.grp[i].outs[j];
-        if (o.kind) info.out[info.n_out++] = span_of(o.ptr, o.ld, g.n, o.kind == 1 ? 1 : o.kind == 2 ? 2 : 4);
+        if (o.kind) { info.out_grp[info.n_out] = i; info.out[info.n_out++] = span_of(o.ptr, o.ld, g.n, o.kind == 1 ? 1 : o.kind == 2 ? 2 : 4); }
       }
       // weights and their scales are never chain outputs in a forward pass; if they were, run apart
       const uint8_t* blo = static_cast<const uint8_t*>(g.b);
@@ -1490,6 +1564,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
         for (int o = 0; o < cs->info[r].n_out; ++o) b_clash = b_clash || overlap(bs, cs->info[r].out[o]);
     }
     int deps[kMaxDeps], n_deps = 0;
+    bool read_grp[kChainMax][kMaxGroups] = {};
     bool clash = b_clash;
     for (int r = 0; r < cs->args.n && !clash; ++r) {
       const ChainRecInfo& E = cs->info[r];
@@ -1499,7 +1574,8 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       }
       bool reads = false;
       for (int x = 0; x < info.n_in; ++x)
-        for (int o = 0; o < E.n_out; ++o) reads = reads || overlap(info.in[x], E.out[o]);
+        for (int o = 0; o < E.n_out; ++o)
+          if (overlap(info.in[x], E.out[o])) { reads = true; read_grp[r][E.out_grp[o]] = true; }
       if (reads) {
         if (n_deps == kMaxDeps) clash = true;
         else deps[n_deps++] = r;
@@ -1511,8 +1587,11 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs, int count, cudaStream_t st) 
       n_deps = 0;
     }
     for (int d = 0; d < kMaxDeps; ++d) p.deps[d] = d < n_deps ? deps[d] : -1;
-    for (int d = 0; d < n_deps; ++d) cs->args.rec[deps[d]].p.signal = 1;
-    p.signal = 0;
+    for (int d = 0; d < n_deps; ++d)
+      for (int i = 0; i < kMaxGroups; ++i)
+        if (read_grp[deps[d]][i]) cs->args.rec[deps[d]].p.grp[i].signal = 1;
+    for (int i = 0; i < kMaxGroups; ++i) p.grp[i].signal = 0;
+    p.need = 0;
     p.stamp = nullptr;
     const int slot = cs->args.n++;
     cs->args.rec[slot].maps = maps;
