@@ -60,8 +60,12 @@ struct OutDesc {
 // column tiles are numbered one after the other, so the persistent CTAs work through all of them
 // and only the first tile's main loop and the last tile's epilogue stay unoverlapped.
 constexpr int kMaxGroups = 3;
-struct GroupMaps { CUtensorMap a, b, om[kNumOuts], fast; };   // fast: the output of a group served by a fast epilogue body
-struct AllMaps { GroupMaps g[kMaxGroups]; };
+// Tensor maps of a record sit in a pool; per group an index row says where its A and B operand
+// maps, the map of the output a fast epilogue body writes and the maps of its outputs are.
+constexpr int kMapsPerGroup = 3 + kNumOuts;
+enum : int { MAP_A = 0, MAP_B = 1, MAP_FAST = 2, MAP_OUT = 3 };
+constexpr int kPoolAll = kMaxGroups * kMapsPerGroup;   // a launch of its own: every map has its place
+constexpr int kPoolChain = 8;                          // a record of a chain: the (distinct) maps it really uses
 // Epilogue bodies.  The general one handles any combination of outputs with run-time branches; the
 // two common combinations have straight-line bodies (same arithmetic, same order).
 enum : int32_t { EPI_GENERAL = 0, EPI_CODES1 = 1, EPI_Y = 2 };
@@ -100,20 +104,21 @@ struct GemmParams {
   ConvDesc conv;              // conv.on: A comes from the gather warps (single-group launches only)
   // chains: records of the same launch whose output rows this record reads (-1: none), and
   // whether a later record of the launch reads this one's
+  uint8_t mi[kMaxGroups][kMapsPerGroup];   // pool indices of the groups' tensor maps
   int32_t deps[kMaxDeps];
   int32_t need;               // finished tiles per row tile and CTA rank that make this record's rows complete for its readers
 };
 // What one launch gets: one record, or a chain of them (see the kernel).
-constexpr int kChainMax = 7;
-struct Rec { AllMaps maps; GemmParams p; };
-template <int N> struct LaunchArgs {
-  Rec rec[N];
+constexpr int kChainMax = 16;
+template <int POOL> struct Rec { CUtensorMap m[POOL]; GemmParams p; };
+template <bool CHAIN> struct LaunchArgs {
+  Rec<CHAIN ? kPoolChain : kPoolAll> rec[CHAIN ? kChainMax : 1];
   int32_t n;             // records in use
   int32_t total_tiles;   // tiles of all records together
   int32_t flag_stride;   // counters per record (two per row tile: one per CTA of the pair)
   unsigned* flags;       // [n x flag_stride], zero when the launch starts
 };
-static_assert(sizeof(LaunchArgs<kChainMax>) <= 32764, "kernel parameters are limited to 32764 bytes");
+static_assert(sizeof(LaunchArgs<true>) <= 32764, "kernel parameters are limited to 32764 bytes");
 
 // ---------------------------------------------------------------------------- PTX wrappers
 
@@ -168,6 +173,7 @@ __device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, v
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (v >= need) return true;
+    __nanosleep(100);        // the warp that polls is ahead of the producer; it need not spin at full rate
     if ((it & 63u) == 0) {
       if (*abort_flag) return false;
       const uint64_t now = global_timer();
@@ -188,6 +194,7 @@ __device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volat
     uint32_t v;
     asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
     if (v >= need) return true;
+    __nanosleep(40);
     if ((it & 1023u) == 0) {
       if (*abort_flag) return false;
       const uint64_t now = global_timer();
@@ -539,7 +546,7 @@ __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUt
 
 // One 32-column chunk of one accumulator row (all 32 lanes of the warp call this together).
 template <bool BF16>
-__device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtensorMap* om, int m, uint32_t epi_bytes,
+__device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtensorMap* pool, const uint8_t* mi, int m, uint32_t epi_bytes,
                                                uint32_t (&v)[32], float cs_lane,
                                                int64_t row, int row0, int col0, uint32_t stage, uint32_t& cursor, int lane) {
   const int ncols = p.n - col0;                    // valid columns in this chunk (may be <= 0 or > 32)
@@ -547,7 +554,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
   const bool row_ok = row < m;
   const bool full = ncols >= 32;
 
-  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &om[0], v, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
+  if (!BF16 && p.outs[0].kind) store_piece<32>(p.outs[0], &pool[mi[MAP_OUT]], v, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
   if (!p.need_y) return;
 
   float y[32];
@@ -588,7 +595,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
     uint32_t w[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(y[i]);
-    store_piece<32>(p.outs[1], &om[1], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
+    store_piece<32>(p.outs[1], &pool[mi[MAP_OUT + 1]], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
   }
 #pragma unroll
   for (int s = 0; s < kMaxSlots; ++s) {
@@ -599,7 +606,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
       for (int i = 0; i < 8; ++i)
         w[i] = pack4(code_word(y[4 * i], o.inv_scale, o.qmax), code_word(y[4 * i + 1], o.inv_scale, o.qmax),
                      code_word(y[4 * i + 2], o.inv_scale, o.qmax), code_word(y[4 * i + 3], o.inv_scale, o.qmax));
-      store_piece<8>(o, &om[2 + s], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
+      store_piece<8>(o, &pool[mi[MAP_OUT + 2 + s]], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
     } else if (o.kind == 2) {
       uint32_t w[16];
 #pragma unroll
@@ -607,7 +614,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
         __nv_bfloat162 h = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
         w[i] = *reinterpret_cast<uint32_t*>(&h);
       }
-      store_piece<16>(o, &om[2 + s], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
+      store_piece<16>(o, &pool[mi[MAP_OUT + 2 + s]], w, row_ok, ncols, row, row0, col0, stage, epi_bytes, cursor, lane);
     }
   }
 }
@@ -627,10 +634,10 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
 // shape, operand type, stage count, staging size, rows and grid.
 template <bool BF16, bool PAIR, bool GROUPED, bool CHAIN>
 __global__ void __launch_bounds__(kGemmThreadsConv, 1)
-gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
+gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
   const GemmParams& p = L.rec[0].p;        // what all records of the launch have in common is read here
   const GemmParams* q = &L.rec[0].p;       // the record this thread's role is working on
-  const AllMaps* mp = &L.rec[0].maps;
+  const CUtensorMap* mp = L.rec[0].m;      // its pool of tensor maps
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the 128B swizzle atoms
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -668,18 +675,18 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
   int num_tiles, step_tn, step_tm, tm0, tn0;
   auto set_record = [&](int li) {
     q = &L.rec[CHAIN ? li : 0].p;
-    mp = &L.rec[CHAIN ? li : 0].maps;
+    mp = L.rec[CHAIN ? li : 0].m;
     num_tiles = q->tiles_m * q->tiles_n;
     step_tn = tile_step / q->tiles_m; step_tm = tile_step - step_tn * q->tiles_m;
     tm0 = tile0 % q->tiles_m; tn0 = tile0 / q->tiles_m;
   };
   set_record(0);
   // chains: position in the launch's tile sequence
-  struct Cur { int li, first, ntiles; const GemmParams* q; const AllMaps* mp; };
+  struct Cur { int li, first, ntiles; const GemmParams* q; const CUtensorMap* mp; };
   auto cur_seek = [&](Cur& c, int g) {       // g < L.total_tiles
     while (g >= c.first + c.ntiles) {
       c.first += c.ntiles; ++c.li;
-      c.q = &L.rec[CHAIN ? c.li : 0].p; c.mp = &L.rec[CHAIN ? c.li : 0].maps;
+      c.q = &L.rec[CHAIN ? c.li : 0].p; c.mp = L.rec[CHAIN ? c.li : 0].m;
       c.ntiles = c.q->tiles_m * c.q->tiles_n;
     }
   };
@@ -706,11 +713,11 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
   uint32_t ld_dst = stage0, ld_bar = full0;      // stage address and its full barrier
   int ld_x = 0, ld_ya = 0, ld_yb = 0;            // TMA coordinates of the next k-block
   int ld_tm = tm0, ld_tn = tn0;
-  const CUtensorMap* ld_map_a = &mp->g[0].a;
-  const CUtensorMap* ld_map_b = &mp->g[0].b;
+  const CUtensorMap* ld_map_a = &mp[q->mi[0][MAP_A]];
+  const CUtensorMap* ld_map_b = &mp[q->mi[0][MAP_B]];
   auto set_tile_coords = [&]() {
     const int g = group_of(ld_tn);
-    if (GROUPED) { ld_map_a = &mp->g[g].a; ld_map_b = &mp->g[g].b; }
+    if (GROUPED) { ld_map_a = &mp[q->mi[g][MAP_A]]; ld_map_b = &mp[q->mi[g][MAP_B]]; }
     ld_ya = ld_tm * rows_per_tile + rank * BM;
     ld_yb = tile_in_group(ld_tn, g) * p.bn + rank * b_rows;
   };
@@ -743,8 +750,8 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
   };
 
   if (threadIdx.x == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&mp->g[0].a) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&mp->g[0].b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&mp[q->mi[0][MAP_A]]) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&mp[q->mi[0][MAP_B]]) : "memory");
     const uint32_t full_count = 1 + (p.conv.on ? kGatherWarps * (PAIR ? 2 : 1) : 0);   // the TMA thread, plus one arrival per gather warp
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
@@ -793,8 +800,8 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
         int gi, tm, tn;
         locate(cq, g - cur.first, gi, tm, tn);
         if (!cleared_wait(cleared_addr, ++t_ld, abort_flag, p.err)) { ok = false; break; }
-        const CUtensorMap* ma = &cur.mp->g[gi].a;
-        const CUtensorMap* mb = &cur.mp->g[gi].b;
+        const CUtensorMap* ma = &cur.mp[cq->mi[gi][MAP_A]];
+        const CUtensorMap* mb = &cur.mp[cq->mi[gi][MAP_B]];
         const int ya = tm * rows_per_tile + rank * BM;
         const int yb = (tn - cq->grp[gi].tn_begin) * p.bn + rank * b_rows;
         int x = 0;
@@ -1082,9 +1089,9 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
             __syncwarp();
           }
           if (G.mode == EPI_CODES1)
-            epilogue_tile_fast<BF16, PAIR, true>(G, &mp->g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
+            epilogue_tile_fast<BF16, PAIR, true>(G, &mp[q->mi[g][MAP_FAST]], tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
           else
-            epilogue_tile_fast<BF16, PAIR, false>(G, &mp->g[g].fast, tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
+            epilogue_tile_fast<BF16, PAIR, false>(G, &mp[q->mi[g][MAP_FAST]], tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
         }
         prev_fast = true;
       } else {
@@ -1105,7 +1112,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN ? kChainMax : 1> L) {
             if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
           }
           const float csl = c ? cs[1] : cs[0];
-          epilogue_chunk<BF16>(G, mp->g[g].om, q->m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
+          epilogue_chunk<BF16>(G, mp, q->mi[g], q->m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
         }
         if (nch == 0) {
           __syncwarp();
@@ -1143,7 +1150,7 @@ struct ChainRecInfo { Span in[2 * kMaxGroups]; int n_in; Span out[kNumOuts * kMa
 constexpr size_t kFlagRingBytes = 8u << 20;
 constexpr int kChainMaxTilesM = 2048;
 struct ChainState {
-  LaunchArgs<kChainMax> args;     // args.n records collected so far
+  LaunchArgs<true> args;          // args.n records collected so far
   ChainRecInfo info[kChainMax];
   double ops = 0.0;
   unsigned* ring = nullptr;       // device counters, handed out front to back and cleared when used up
@@ -1310,7 +1317,7 @@ int gemm_chain_flush(Ctx* ctx) {
   if (!cs || cs->args.n == 0) return QCFG_OK;
   const int n = cs->args.n;
   cs->args.n = 0;
-  LaunchArgs<kChainMax>& A = cs->args;
+  LaunchArgs<true>& A = cs->args;
   // counters: two per row tile and record, from a region nobody has used since it was cleared
   const int stride = 2 * A.rec[0].p.tiles_m;
   const size_t need = (size_t)n * stride * sizeof(unsigned);
@@ -1444,8 +1451,10 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
   p.idesc = ((g0.is_bf16 ? 1u : 2u) << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(tile_rows >> 4) << 24);
   p.err = err_word(ctx);
 
-  AllMaps maps;
-  memset(&maps, 0, sizeof(maps));
+  CUtensorMap maps[kPoolAll];      // group i's maps at i * kMapsPerGroup + MAP_*
+  memset(maps, 0, sizeof(maps));
+  for (int i = 0; i < kMaxGroups; ++i)
+    for (int j = 0; j < kMapsPerGroup; ++j) p.mi[i][j] = (uint8_t)(i * kMapsPerGroup + j);
   bool wide = false;
   int32_t tn_total = 0;
   double ops = 0.0;
@@ -1473,16 +1482,16 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
     if (!G.need_y && !G.outs[0].kind) return set_error(ctx, QCFG_EINVAL, "gemm: no output requested");
     if (G.need_y && !g.is_bf16 && !g.scale_w) return set_error(ctx, QCFG_EINVAL, "gemm: scale_w is null");
     for (int j = 0; j < kNumOuts; ++j)
-      if (G.outs[j].kind) G.outs[j].tma = make_out_map(&maps.g[i].om[j], G.outs[j], g.m, g.n) ? 1 : 0;
+      if (G.outs[j].kind) G.outs[j].tma = make_out_map(&maps[i * kMapsPerGroup + MAP_OUT + j], G.outs[j], g.m, g.n) ? 1 : 0;
     // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
     for (int j = 0; j < kNumOuts; ++j) if (G.outs[j].kind >= 2 && G.outs[j].tma) wide = true;
     G.mode = EPI_GENERAL;
     if (bn == 256 && !G.residual && !G.outs[0].kind && !G.outs[3].kind && !G.outs[4].kind) {
-      if (!G.outs[1].kind && G.outs[2].kind == 1 && make_fast_map(&maps.g[i].fast, G.outs[2], g.m, g.n)) G.mode = EPI_CODES1;
-      else if (G.outs[1].kind && !G.outs[2].kind && make_fast_map(&maps.g[i].fast, G.outs[1], g.m, g.n)) { G.mode = EPI_Y; wide = true; }
+      if (!G.outs[1].kind && G.outs[2].kind == 1 && make_fast_map(&maps[i * kMapsPerGroup + MAP_FAST], G.outs[2], g.m, g.n)) G.mode = EPI_CODES1;
+      else if (G.outs[1].kind && !G.outs[2].kind && make_fast_map(&maps[i * kMapsPerGroup + MAP_FAST], G.outs[1], g.m, g.n)) { G.mode = EPI_Y; wide = true; }
     }
-    int rc = g.conv_kh > 0 ? QCFG_OK : make_map(ctx, &maps.g[i].a, g.a, g.is_bf16, g.k, g.m, g.lda, BM);
-    if (rc == QCFG_OK) rc = make_map(ctx, &maps.g[i].b, g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
+    int rc = g.conv_kh > 0 ? QCFG_OK : make_map(ctx, &maps[i * kMapsPerGroup + MAP_A], g.a, g.is_bf16, g.k, g.m, g.lda, BM);
+    if (rc == QCFG_OK) rc = make_map(ctx, &maps[i * kMapsPerGroup + MAP_B], g.b, g.is_bf16, g.k, g.n, g.ldb, pair ? bn / 2 : bn);
     if (rc != QCFG_OK) return rc;
     ops += 2.0 * (double)g.m * (double)g.n * (double)g.k;
   }
@@ -1533,13 +1542,46 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
     if (grid > 2 * num_tiles && !chainable) grid = 2 * num_tiles;
   } else if (grid > num_tiles) grid = num_tiles;
   const size_t smem = (size_t)kSmemHeader + kCsBytes + 1024 + (size_t)kEpiWarps * p.epi_bytes + (size_t)stages * stage_bytes;
+  // a chain record carries only the distinct maps it uses; one that needs more runs on its own
+  CUtensorMap pool[kPoolChain];
+  bool fits = true;
+  if (chainable) {
+    memset(pool, 0, sizeof(pool));
+    int used = 0;
+    auto place = [&](int i, int j) {
+      const CUtensorMap& mm = maps[i * kMapsPerGroup + j];
+      int at = -1;
+      for (int u = 0; u < used && at < 0; ++u) if (memcmp(&pool[u], &mm, sizeof(CUtensorMap)) == 0) at = u;
+      if (at < 0) {
+        if (used == kPoolChain) { fits = false; return; }
+        pool[used] = mm; at = used++;
+      }
+      p.mi[i][j] = (uint8_t)at;
+    };
+    for (int i = 0; i < kMaxGroups; ++i)
+      for (int j = 0; j < kMapsPerGroup; ++j) p.mi[i][j] = 0;
+    for (int i = 0; i < count && fits; ++i) {
+      place(i, MAP_A);
+      place(i, MAP_B);
+      if (p.grp[i].mode != EPI_GENERAL) {       // a fast body writes through this one map only
+        place(i, MAP_FAST);
+        continue;
+      }
+      for (int j = 0; j < kNumOuts && fits; ++j)
+        if (p.grp[i].outs[j].kind && p.grp[i].outs[j].tma) place(i, MAP_OUT + j);
+    }
+    if (!fits)
+      for (int i = 0; i < kMaxGroups; ++i)
+        for (int j = 0; j < kMapsPerGroup; ++j) p.mi[i][j] = (uint8_t)(i * kMapsPerGroup + j);
+  }
+  const bool chained = chainable && fits;
   if (cs && cs->args.n > 0 &&
-      (!chainable || cs->args.n == kChainMax || cs->st != st || cs->bf16 != (g0.is_bf16 != 0) || cs->grid != grid ||
+      (!chained || cs->args.n == kChainMax || cs->st != st || cs->bf16 != (g0.is_bf16 != 0) || cs->grid != grid ||
        cs->smem != smem || cs->m != g0.m)) {
     const int rc = gemm_chain_flush(ctx);
     if (rc != QCFG_OK) return rc;
   }
-  if (chainable) {
+  if (chained) {
     // What the record reads and writes, as byte ranges.  Reading rows an earlier record of the
     // chain writes is a dependency the kernel waits for; any other overlap ends the chain first.
     ChainRecInfo info{};
@@ -1594,7 +1636,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
     p.need = 0;
     p.stamp = nullptr;
     const int slot = cs->args.n++;
-    cs->args.rec[slot].maps = maps;
+    memcpy(cs->args.rec[slot].m, pool, sizeof(pool));
     cs->args.rec[slot].p = p;
     cs->info[slot] = info;
     cs->ops += ops;
@@ -1617,15 +1659,15 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
   attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 2 : 1;
-  using Kern = void (*)(const LaunchArgs<1>);
+  using Kern = void (*)(const LaunchArgs<false>);
   static const Kern kernels[8] = {
       gemm_kernel<false, false, false, false>, gemm_kernel<false, false, true, false>, gemm_kernel<false, true, false, false>,
       gemm_kernel<false, true, true, false>,   gemm_kernel<true, false, false, false>,  gemm_kernel<true, false, true, false>,
       gemm_kernel<true, true, false, false>,   gemm_kernel<true, true, true, false>};
   const Kern kern = kernels[(g0.is_bf16 ? 4 : 0) + (pair ? 2 : 0) + (count > 1 ? 1 : 0)];
   p.stamp = prof_stamp(ctx, g0.is_bf16 ? 1 : 0, ops);
-  static thread_local LaunchArgs<1> one;
-  one.rec[0].maps = maps;
+  static thread_local LaunchArgs<false> one;
+  memcpy(one.rec[0].m, maps, sizeof(maps));
   one.rec[0].p = p;
   one.n = 1; one.total_tiles = num_tiles; one.flag_stride = 0; one.flags = nullptr;
   prof_begin(ctx, g0.is_bf16 ? 1 : 0, st);
