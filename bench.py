@@ -35,9 +35,13 @@ UNIT = "evals/s"
 N_EVALS = 72
 TOKENS = 32 * 384
 WORKLOAD = "bert_base_x12_sweep_calibrate_greedy72"
-# DRAM bytes (read + write) per int8 GEMM launch from the ncu capture summarised in
-# profiles/gemm_int8_bert_base_block.md; set to None whenever the GEMM kernel changes.
-GEMM_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) per int8 GEMM of a BERT-base block at 12288 tokens (mean of the four:
+# q/k/v grouped, o, ffn1, ffn2) from the ncu capture summarised in
+# profiles/gemm_int8_bert_base_block.md, taken with one launch per GEMM (ncu cannot launch the
+# cooperative chain kernel); a chained launch is charged this figure times the GEMMs it runs.
+# Set to None whenever the GEMM kernel changes.
+GEMM_TRAFFIC_BYTES = 27.1e6
+GEMMS_PER_EVAL = 48          # 12 blocks x (q+k+v grouped, o, ffn1, ffn2)
 DATASHEET_INT8_TOPS = 4500.0      # B200 dense int8, vendor datasheet (an outside figure)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -336,6 +340,7 @@ def run_gpu(args):
         torch.cuda.set_device(0)
     dev_index = torch.cuda.current_device()
     ctx = q.Context(dev_index)
+    ctx.set_gemm_chains(not args.no_chains)
     peaks = load_peaks()
 
     w = wl.bert_base_x12()
@@ -521,7 +526,7 @@ def run_gpu(args):
                        "parallelism": "replicas" if world > 1 else "single"},
             "clocks": clocks, "gpu_launches": int(launches),
             "host": {"enqueue_ms_per_eval": host_enqueue_ms, "device_ms_per_eval": ms_total / args.steps / N_EVALS,
-                     "note": "host time of one qcfg_eval_config call (planning, tensor maps, 48 GEMM records in 7 chained launches) against the device time it hides behind"},
+                     "note": "host time of one qcfg_eval_config call (planning, tensor maps, 48 GEMMs in 3 chained launches) against the device time it hides behind"},
             "e2e": e2e, "launches_before_timed": int(launches0),
             "roofline": {"kernel": "gemm_kernel<int8>", "bound": "tensor", "achieved": achieved, "peak": sustained2,
                          "unit": "TOP/s", "frac": achieved / sustained2,
@@ -531,12 +536,15 @@ def run_gpu(args):
                                                        "own_large_square_int8": own},
                          "launches": int(g_n), "avg_launch_us": 1e3 * g_ms / max(g_n, 1),
                          "kernel_ms_per_step": g_ms / args.steps, "bf16_kernel_ms_per_step": b_ms / args.steps,
-                         "traffic": GEMM_TRAFFIC_BYTES,
+                         "traffic": None if GEMM_TRAFFIC_BYTES is None or not g_n else
+                                    GEMM_TRAFFIC_BYTES * GEMMS_PER_EVAL * N_EVALS * args.steps / g_n,
                          "traffic_source": "none: the kernel changed after the last ncu capture" if GEMM_TRAFFIC_BYTES is None else
-                                           "ncu dram bytes per launch (a chain of layers' GEMMs at 12288 tokens)",
+                                           "ncu dram bytes per GEMM (mean of the four GEMMs of one block at 12288 tokens, one launch per GEMM: "
+                                           "ncu cannot launch the cooperative chain kernel) x GEMMs per timed launch",
+                         "gemms_per_launch": GEMMS_PER_EVAL * N_EVALS * args.steps / max(g_n, 1),
                          "how": "the timed pass that gives `value`: every CTA folds %globaltimer after its wait for the "
                                 "previous kernel and at its end into the launch's slot; duration = last end - first start; "
-                                "a launch is a chain of up to seven consecutive layers' GEMMs",
+                                "a launch is a chain of up to sixteen consecutive GEMMs",
                          "event_pass": {"int8_gemm_avg_launch_us": 1e3 * eg_ms / max(eg_n, 1),
                                         "tops": eg_ops / (eg_ms * 1e-3) / 1e12 if eg_ms else None,
                                         "share_of_kernel_time": eg_ms / max(eg_ms + eb_ms + eo_ms, 1e-9),
@@ -573,6 +581,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used when profiling)")
     ap.add_argument("--no-workloads", action="store_true", help="skip the short legs of the other four workloads")
+    ap.add_argument("--no-chains", action="store_true",
+                    help="one launch per GEMM instead of chained launches (ncu cannot launch the cooperative chain kernel)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -111,7 +111,7 @@ int qcfg_set_implicit_conv(qcfg_ctx* ctx, int enabled);
 /* Switches chained GEMM launches in model evaluations (default on): consecutive GEMMs of a
  * forward pass that use the two-CTA 256-column tiles, share rows and operand type and need no
  * other kernel in between (their operands come out of the producers' epilogues) run as ONE
- * cooperative launch of up to seven layers.  Its CTA pairs work through the tiles of all layers
+ * cooperative launch of up to sixteen GEMMs.  Its CTA pairs work through the tiles of all layers
  * in one sequence; a tile starts once the row tiles it reads have been completed (per-row-tile
  * counters in device memory, every wait bounded).  Off: one launch per GEMM (or per group of
  * independent GEMMs).  Results are bit-identical either way.                                  */

@@ -33,6 +33,7 @@ def main():
     ap.add_argument("--latency", type=int, default=0, help="repetitions: print the per-width latency table sums and model sizes")
     ap.add_argument("--noise", type=float, default=0.0, help="lambda: run the noise-injection sensitivity E_N over all layers")
     ap.add_argument("--no-grouping", action="store_true", help="one launch per layer")
+    ap.add_argument("--no-chains", action="store_true", help="one launch per GEMM instead of chained launches")
     ap.add_argument("--single-cta", action="store_true", help="128-row GEMM tiles on one CTA each instead of CTA pairs")
     args = ap.parse_args()
 
@@ -44,6 +45,7 @@ def main():
     ctx = Context(0)
     ctx.set_pair_tiles(not args.single_cta)
     ctx.set_grouping(not args.no_grouping)
+    ctx.set_gemm_chains(not args.no_chains)
     weights = [torch.from_numpy(a).cuda() for a in w.weights]
     x = torch.from_numpy(w.x).cuda()
     model = Model(ctx, w.layers, weights)
