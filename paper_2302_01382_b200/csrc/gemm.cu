@@ -208,6 +208,27 @@ __device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volat
   }
 }
 
+// Chains: waits (whole warp) until every epilogue warp has reported `need` tiles; lane w reads warp w's counter.
+__device__ __forceinline__ bool reported_wait(uint32_t rep0, uint32_t need, int lane, volatile int* abort_flag, unsigned* err) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    uint32_t v = need;
+    if (lane < kEpiWarps) asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(rep0 + 4 * lane) : "memory");
+    if (__all_sync(0xffffffffu, v >= need)) return true;
+    __nanosleep(40);
+    if ((it & 1023u) == 0) {
+      bool give_up = *abort_flag != 0;
+      const uint64_t now = global_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
+        if (lane == 0) { atomicOr(err, ERR_TIMEOUT); *abort_flag = 1; }
+        give_up = true;
+      }
+      if (__any_sync(0xffffffffu, give_up)) return false;
+    }
+  }
+}
+
 // The same wait for a whole converged warp, written so that the compiler sees warp-uniform control
 // flow (the spin is inside one asm statement, the outcome is a vote): the producer and the MMA
 // issuer run their loops on all 32 lanes, which keeps their address and descriptor arithmetic on
@@ -475,13 +496,13 @@ __device__ __forceinline__ float2 code_words2(float2 y, float2 inv2, float qmax)
 // written by one TMA store.  Otherwise the fp32 matrix, each 32 x 32 block staged in 128-byte
 // rows (128B swizzle), one TMA store per block; the single staging slot is reused once the
 // previous store has read it.
-// done_bar (chains, else 0): barrier to arrive on once the stores this warp issued for its previous
-// tile have completed; that is checked after this tile's first piece, a quarter of an epilogue
-// after they were issued.
+// rep_addr (chains, else 0): this warp's report counter in shared memory, set to rep_val once the
+// stores the warp issued for its previous tile have completed; that is checked after this tile's
+// first piece, a quarter of an epilogue after they were issued.
 template <bool BF16, bool PAIR, bool CODES>
 __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUtensorMap* fmap, uint32_t tbase,
                                                    const float* cs, uint32_t stage, int row0, int col0, int lane,
-                                                   uint32_t tempty_bar, uint32_t done_bar) {
+                                                   uint32_t tempty_bar, uint32_t rep_addr, uint32_t rep_val) {
   const int act = G.act;
   const float qmax = G.outs[2].qmax;
   const float2 inv2 = make_float2(G.outs[2].inv_scale, G.outs[2].inv_scale);
@@ -518,9 +539,9 @@ __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUt
       __syncwarp();
     }
     piece(va, 2 * h);
-    if (h == 0 && done_bar && lane == 0) {    // a quarter of a tile after the previous tile's last store
+    if (h == 0 && rep_addr && lane == 0) {    // a quarter of a tile after the previous tile's last store
       asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-      mbar_arrive(done_bar);
+      asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(rep_addr), "r"(rep_val) : "memory");
     }
     tmem_ld_wait();
     if (h == 0) {
@@ -545,7 +566,7 @@ __device__ __forceinline__ void epilogue_tile_fast(const GroupDesc& G, const CUt
 }
 
 // One 32-column chunk of one accumulator row (all 32 lanes of the warp call this together).
-template <bool BF16>
+template <bool BF16, bool CHAIN>
 __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtensorMap* pool, const uint8_t* mi, int m, uint32_t epi_bytes,
                                                uint32_t (&v)[32], float cs_lane,
                                                int64_t row, int row0, int col0, uint32_t stage, uint32_t& cursor, int lane) {
@@ -568,12 +589,14 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
       y[i] = __fmul_rn((float)(int32_t)v[i], __shfl_sync(0xffffffffu, cs_lane, i));
   }
   if (p.residual && row_ok) {
-    // read through L2: in a chain another SM may have written the shortcut earlier in this launch
+    // In a chain another SM may have written the shortcut earlier in this launch, so it is read
+    // with ordinary loads, not through the read-only path.  (A stale L1 line is impossible: within a
+    // launch every address is written at most once and read only after that write has been seen.)
     const float* r = p.residual + row * p.ldr + col0;
     if (full && (p.ldr & 3) == 0 && (((uintptr_t)p.residual) & 15) == 0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        float4 r4 = __ldcg(reinterpret_cast<const float4*>(r) + i);
+        const float4 r4 = CHAIN ? *(reinterpret_cast<const float4*>(r) + i) : __ldg(reinterpret_cast<const float4*>(r) + i);
         y[4 * i + 0] = __fadd_rn(y[4 * i + 0], r4.x);
         y[4 * i + 1] = __fadd_rn(y[4 * i + 1], r4.y);
         y[4 * i + 2] = __fadd_rn(y[4 * i + 2], r4.z);
@@ -581,7 +604,7 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
       }
     } else {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) if (i < ncols) y[i] = __fadd_rn(y[i], __ldcg(r + i));
+      for (int i = 0; i < 32; ++i) if (i < ncols) y[i] = __fadd_rn(y[i], CHAIN ? r[i] : __ldg(r + i));
     }
   }
   if (p.act == QCFG_ACT_RELU) {
@@ -660,7 +683,9 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
   const uint32_t stage_bytes = (uint32_t)(BM + b_rows) * kStageKBytes;
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMaxStages;
   const uint32_t tfull0 = empty0 + 8 * kMaxStages, tempty0 = tfull0 + 16;
-  const uint32_t done0 = tempty0 + 16;           // chains: done[4], the epilogue warps' stores of a tile have completed
+  // chains: per epilogue warp, the number of its tiles whose stores have completed (counters, not
+  // phase barriers: the warp that reads them may fall any number of tiles behind)
+  const uint32_t rep0 = smem_u32(smem + 320);
   const int tile0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // first tile of this CTA (pair)
   const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int rows_per_tile = PAIR ? 2 * BM : BM;
@@ -755,7 +780,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
     const uint32_t full_count = 1 + (p.conv.on ? kGatherWarps * (PAIR ? 2 : 1) : 0);   // the TMA thread, plus one arrival per gather warp
     for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, full_count); mbar_init(empty0 + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, PAIR ? 2 * kEpiWarps : kEpiWarps); }
-    if (CHAIN) for (int a = 0; a < 4; ++a) mbar_init(done0 + 8 * a, kEpiWarps);
+    if (CHAIN) for (int a = 0; a < kEpiWarps; ++a) *reinterpret_cast<volatile uint32_t*>(smem + 320 + 4 * a) = 0u;
     *abort_flag = 0;
     *reinterpret_cast<volatile uint32_t*>(smem + 264) = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -888,7 +913,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
       int t = 0;
       for (int g = tile0; g < total_tiles; g += tile_step, ++t) {
         cur_seek(cur, g);
-        if (!mbar_wait_warp(done0 + 8 * (t & 3), (uint32_t)(t >> 2) & 1u, abort_flag, p.err)) break;
+        if (!reported_wait(rep0, (uint32_t)t + 1u, lane, abort_flag, p.err)) break;
         int gi, tm, tn;
         locate(cur.q, g - cur.first, gi, tm, tn);
         if (elected && cur.q->grp[gi].signal) {
@@ -1061,15 +1086,15 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
       // accumulator is already there the check is left to the body (after its first piece, when
       // the old stores have landed); when it is not, this tile may itself be waiting for
       // rows other CTAs produce, and they for the report, so the report goes out now.
-      uint32_t done_bar = (CHAIN && t > 0) ? done0 + 8 * ((t - 1) & 3) : 0u;
+      uint32_t rep_addr = (CHAIN && t > 0) ? rep0 + 4 * ew : 0u;
       const bool fast_inside = G.mode != EPI_GENERAL && !(row0 >= q->m || col_base >= G.n);
-      if (done_bar && !(fast_inside && __all_sync(0xffffffffu, mbar_try_wait(tfull0 + 8 * a, (t >> 1) & 1)))) {
+      if (rep_addr && !(fast_inside && __all_sync(0xffffffffu, mbar_try_wait(tfull0 + 8 * a, (t >> 1) & 1)))) {
         if (lane == 0) {
           asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-          mbar_arrive(done_bar);
+          asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(rep_addr), "r"((uint32_t)t) : "memory");
         }
         __syncwarp();
-        done_bar = 0;
+        rep_addr = 0;
       }
       if (!mbar_wait(tfull0 + 8 * a, (t >> 1) & 1, abort_flag, p.err)) { ok = false; break; }
       tc_fence_after();
@@ -1089,9 +1114,9 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
             __syncwarp();
           }
           if (G.mode == EPI_CODES1)
-            epilogue_tile_fast<BF16, PAIR, true>(G, &mp[q->mi[g][MAP_FAST]], tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
+            epilogue_tile_fast<BF16, PAIR, true>(G, &mp[q->mi[g][MAP_FAST]], tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, rep_addr, (uint32_t)t);
           else
-            epilogue_tile_fast<BF16, PAIR, false>(G, &mp[q->mi[g][MAP_FAST]], tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, done_bar);
+            epilogue_tile_fast<BF16, PAIR, false>(G, &mp[q->mi[g][MAP_FAST]], tbase, cs_tab, stage, row0, col_base, lane, tempty_bar, rep_addr, (uint32_t)t);
         }
         prev_fast = true;
       } else {
@@ -1112,7 +1137,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
             if (lane == 0) { if (PAIR) mbar_arrive_leader(tempty_bar); else mbar_arrive(tempty_bar); }
           }
           const float csl = c ? cs[1] : cs[0];
-          epilogue_chunk<BF16>(G, mp, q->mi[g], q->m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
+          epilogue_chunk<BF16, CHAIN>(G, mp, q->mi[g], q->m, (uint32_t)p.epi_bytes, v, csl, row, row0, col_base + 32 * c, stage, cursor, lane);
         }
         if (nch == 0) {
           __syncwarp();
@@ -1124,7 +1149,7 @@ gemm_kernel(const __grid_constant__ LaunchArgs<CHAIN> L) {
     if (CHAIN && t > 0 && ok) {       // the last tile: report it as soon as its stores have completed
       if (lane == 0) {
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        mbar_arrive(done0 + 8 * ((t - 1) & 3));
+        asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(rep0 + 4 * ew), "r"((uint32_t)t) : "memory");
       }
     }
     // all TMA stores of this warp must have completed before the CTA's shared memory goes away
@@ -1151,6 +1176,11 @@ constexpr size_t kFlagRingBytes = 8u << 20;
 constexpr int kChainMaxTilesM = 2048;
 struct ChainState {
   LaunchArgs<true> args;          // args.n records collected so far
+  // the first record once more, set up as a launch of its own: a chain that ends with one record
+  // goes out that way (the cooperative launch only pays when tiles of several GEMMs can overlap)
+  LaunchArgs<false> solo;
+  int solo_grid = 0, solo_grouped = 0;
+  size_t solo_smem = 0;
   ChainRecInfo info[kChainMax];
   double ops = 0.0;
   unsigned* ring = nullptr;       // device counters, handed out front to back and cleared when used up
@@ -1161,7 +1191,7 @@ struct ChainState {
   int64_t m = 0;
   size_t smem = 0;
   cudaStream_t st = nullptr;
-  ChainState() { memset(&args, 0, sizeof(args)); }
+  ChainState() { memset(&args, 0, sizeof(args)); memset(&solo, 0, sizeof(solo)); }
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1318,6 +1348,30 @@ int gemm_chain_flush(Ctx* ctx) {
   const int n = cs->args.n;
   cs->args.n = 0;
   LaunchArgs<true>& A = cs->args;
+  if (n == 1) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cs->solo_grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = cs->solo_smem;
+    cfg.stream = cs->st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cs->solo.rec[0].p.stamp = prof_stamp(ctx, cs->bf16 ? 1 : 0, cs->ops);
+    cs->ops = 0.0;
+    cudaError_t le;
+    if (cs->bf16) le = cs->solo_grouped ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, true, true, false>, cs->solo)
+                                        : cudaLaunchKernelEx(&cfg, gemm_kernel<true, true, false, false>, cs->solo);
+    else le = cs->solo_grouped ? cudaLaunchKernelEx(&cfg, gemm_kernel<false, true, true, false>, cs->solo)
+                               : cudaLaunchKernelEx(&cfg, gemm_kernel<false, true, false, false>, cs->solo);
+    if (le != cudaSuccess) return check_cuda(ctx, le, "gemm launch");
+    count_launch(ctx);
+    return check_cuda(ctx, cudaGetLastError(), "gemm launch");
+  }
   // counters: two per row tile and record, from a region nobody has used since it was cleared
   const int stride = 2 * A.rec[0].p.tiles_m;
   const size_t need = (size_t)n * stride * sizeof(unsigned);
@@ -1511,7 +1565,10 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
   // Launches that may join a chain all take the larger staging size, so any sequence of them
   // shares one shared-memory layout.
   ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
-  const bool chainable = cs && cs->open && pair && !conv && bn == 256 && prof_mode(ctx) != 1 && p.tiles_m <= kChainMaxTilesM;
+  // (a GEMM with fewer tiles than CTA pairs has nothing to overlap with: the wait for its
+  // producer's rows would cost more than the launch boundary it saves)
+  const bool chainable = cs && cs->open && pair && !conv && bn == 256 && prof_mode(ctx) != 1 && p.tiles_m <= kChainMaxTilesM &&
+                         2 * p.tiles_m * p.tiles_n >= sm_count(ctx);
   p.epi_bytes = (wide || chainable) ? 4096 : 2048;
   int stages = (kSmemMax - kSmemHeader - kCsBytes - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
@@ -1636,6 +1693,21 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
     p.need = 0;
     p.stamp = nullptr;
     const int slot = cs->args.n++;
+    if (slot == 0) {
+      GemmParams ps = p;
+      for (int i = 0; i < kMaxGroups; ++i)
+        for (int j = 0; j < kMapsPerGroup; ++j) ps.mi[i][j] = (uint8_t)(i * kMapsPerGroup + j);
+      ps.epi_bytes = wide ? 4096 : 2048;
+      int st_solo = (kSmemMax - kSmemHeader - kCsBytes - 1024 - kEpiWarps * ps.epi_bytes) / stage_bytes;
+      if (st_solo > kMaxStages) st_solo = kMaxStages;
+      ps.stages = st_solo;
+      memcpy(cs->solo.rec[0].m, maps, sizeof(maps));
+      cs->solo.rec[0].p = ps;
+      cs->solo.n = 1; cs->solo.total_tiles = num_tiles; cs->solo.flag_stride = 0; cs->solo.flags = nullptr;
+      cs->solo_grid = grid > 2 * num_tiles ? 2 * num_tiles : grid;
+      cs->solo_grouped = count > 1 ? 1 : 0;
+      cs->solo_smem = (size_t)kSmemHeader + kCsBytes + 1024 + (size_t)kEpiWarps * ps.epi_bytes + (size_t)st_solo * stage_bytes;
+    }
     memcpy(cs->args.rec[slot].m, pool, sizeof(pool));
     cs->args.rec[slot].p = p;
     cs->info[slot] = info;

@@ -283,10 +283,11 @@ def test_implicit_and_materialised_convolutions_agree_bitwise(ctx, fuse):
         model.close()
 
 
-@pytest.mark.parametrize("m", [1664, 700])
+@pytest.mark.parametrize("m", [19200, 19000])
 def test_chained_and_separate_launches_agree_bitwise(ctx, m):
-    """A forward pass whose GEMMs go to the device as chains (one cooperative launch for up to seven
-    consecutive layers, tiles started by per-row-tile counters) gives the same bits as one launch
+    """A forward pass whose GEMMs go to the device as chains (one cooperative launch for up to sixteen
+    consecutive GEMMs, tiles started by per-row-tile counters; a GEMM joins a chain only if it has at
+    least one tile per CTA pair, hence the row counts) gives the same bits as one launch
     per GEMM: all-int8, a mix with 4-bit and 16-bit layers (both operand types chain), every
     output requested (general epilogue) and only the last one (fast epilogue bodies), whole and
     ragged last row tiles.  The launch counter shows that the chains were in fact used."""
