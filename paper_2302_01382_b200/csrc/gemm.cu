@@ -15,8 +15,11 @@
 //               tile's main loop.
 //   warps 18,19 (convolution launches only, 640 threads) gather the A tile of an implicit-GEMM
 //               convolution from the NHWC codes of the layer's input with cp.async.
-// Every mbarrier wait is bounded: after ~2 s it sets the context's error word and the CTA
-// leaves through the normal teardown (TMEM is freed).
+//   warps 18,19 (chained launches only, 640 threads) publish finished tiles (18) and clear tiles
+//               whose input rows are complete (19): a chain runs up to 16 consecutive GEMMs of a
+//               forward pass as one cooperative launch (see the kernel).
+// Every wait (mbarrier, counter in shared or global memory) is bounded: after ~2 s it sets the
+// context's error word and the CTA leaves through the normal teardown (TMEM is freed).
 #include <cuda.h>
 
 #include <cstring>
