@@ -393,7 +393,32 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     const int b = S.bits;
     if (!dirty[l]) continue;
     for (int pl : pending_layers)
-      if (d.src == pl || d.residual_from == pl) { const int frc = flush(); if (frc) return frc; break; }
+      if (d.src == pl || d.residual_from == pl) {
+        // With chained launches the order of independent GEMMs is a free choice, and the best
+        // one keeps a GEMM away from the one it reads: only the layers this one reads go out
+        // now, with half of the others behind them as a buffer; the rest wait and are launched
+        // behind this layer (q, k, v, o: [v, q] now, then [o, k]).
+        if (ctx->chain && pending.size() > 1) {
+          std::vector<GemmArgs> now, later;
+          std::vector<int> now_l, later_l;
+          for (size_t i = 0; i < pending.size(); ++i)
+            if (d.src == pending_layers[i] || d.residual_from == pending_layers[i]) { now.push_back(pending[i]); now_l.push_back(pending_layers[i]); }
+          size_t others = pending.size() - now.size(), taken = 0;
+          for (size_t i = 0; i < pending.size(); ++i) {
+            if (d.src == pending_layers[i] || d.residual_from == pending_layers[i]) continue;
+            if (taken < (others + 1) / 2) { now.push_back(pending[i]); now_l.push_back(pending_layers[i]); ++taken; }
+            else { later.push_back(pending[i]); later_l.push_back(pending_layers[i]); }
+          }
+          const int frc = launch_gemm_group(ctx, now.data(), (int)now.size(), st);
+          if (frc) return frc;
+          pending.swap(later);
+          pending_layers.swap(later_l);
+        } else {
+          const int frc = flush();
+          if (frc) return frc;
+        }
+        break;
+      }
     int rc = ensure_weight_codes(ctx, S, b, st);
     if (rc) return rc;
     // optional per-layer timing: everything this layer launches (operand preparation and GEMM)

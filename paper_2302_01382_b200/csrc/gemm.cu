@@ -1449,10 +1449,10 @@ bool gemm_groupable(const GemmArgs& a, const GemmArgs& b) {
 
 int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t st) {
   if (count < 1 || count > kMaxGroups) return set_error(ctx, QCFG_EINVAL, "gemm: %d groups", count);
-  // While launches are being chained a record's tiles run group after group.  Groups that write
-  // operand codes for later layers go in the middle: the groups before them give the previous
-  // record time to complete the rows they read, the groups after them give their own rows time to
-  // complete before the next record asks for them.
+  // While launches are being chained a record's tiles run group after group.  Of three groups,
+  // those that write operand codes for later layers go in the middle: the group before them gives
+  // the previous record time to complete the rows they read, the group after them gives their own
+  // rows time to complete before the next record asks for them.  Of two, they go first.
   GemmArgs ordered[kMaxGroups];
   {
     ChainState* st_ = static_cast<ChainState*>(chain_slot(ctx));
@@ -1464,7 +1464,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
         if (feeds) feed[n_feed++] = i; else rest[n_rest++] = i;
       }
       int k = 0;
-      const int before = (n_rest + 1) / 2;
+      const int before = count == 3 ? (n_rest + 1) / 2 : 0;   // two groups: the feeder first, the other one is the buffer
       for (int i = 0; i < before; ++i) ordered[k++] = gs_in[rest[i]];
       for (int i = 0; i < n_feed; ++i) ordered[k++] = gs_in[feed[i]];
       for (int i = before; i < n_rest; ++i) ordered[k++] = gs_in[rest[i]];
