@@ -375,6 +375,12 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     S.bits = calibrate ? 16 : bits[l];
   }
   M->reuse_valid = false;                            // until this evaluation has been enqueued completely
+  if (calibrate) {
+    // maxima are folded into the table by atomic max, from epilogues as well: start from zero
+    const int zrc = check_cuda(ctx, cudaMemsetAsync(M->act_absmax_dev.p, 0, (size_t)n * 4, st), "calibration table clear");
+    if (zrc) return zrc;
+    std::fill(M->calib_same_as.begin(), M->calib_same_as.end(), -1);
+  }
   // GEMMs that are ready together and have the same m, k, operand type and tile width (the three
   // projections of an attention block) are collected and launched as one grouped kernel.
   std::vector<GemmArgs> pending;
@@ -541,14 +547,15 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
     }
     // fused re-quantize outputs for consumers whose input is this whole output
     bool all_fused = !S.consumers.empty();
-    int nslots = 0;
+    int nslots = 0, first_ranged = -1;
     for (int c : S.consumers) {
       LayerState& C = M->L[c];
       const int cb = calibrate ? 16 : bits[c];
       // a consumer whose operand is this whole output: a plain row read, or a convolution the GEMM gathers for
       const bool c_implicit = ctx->implicit && !calibrate && implicit_capable(C.d) && C.d.pool_before == QCFG_POOL_NONE;
-      const bool fusable = ctx->fuse && !calibrate && C.d.src_col0 == 0 &&
-                           ((reads_rows_directly(C.d) && C.d.k_in == S.d.n_out) || (c_implicit && C.d.in_c == S.d.n_out));
+      // (in the calibration forward the epilogue also takes the range of what the consumer reads)
+      const bool fusable = ctx->fuse && C.d.src_col0 == 0 &&
+                           ((reads_rows_directly(C.d) && C.d.k_in == S.d.n_out) || (!calibrate && c_implicit && C.d.in_c == S.d.n_out));
       if (!fusable) { all_fused = false; continue; }
       const int64_t c_ld = c_implicit ? C.d.in_c : C.ldk;
       float csc = 1.0f, cinv = 1.0f;
@@ -574,6 +581,10 @@ int forward(Ctx* ctx, Model* M, const uint8_t* bits, const float* x_dev, int64_t
       C.a_ready = true;
       C.bits = cb;
       C.implicit = c_implicit;
+      if (calibrate) {      // one maximum per output tensor; further readers of it take the first one's
+        if (!g.amax) { g.amax = (float*)M->act_absmax_dev.p + c; first_ranged = c; M->calib_same_as[c] = -1; }
+        else M->calib_same_as[c] = first_ranged;
+      }
     }
     float* y_out = (y_dev && y_dev[l]) ? y_dev[l] : nullptr;
     const bool need_y = y_out || !all_fused || S.feeds_residual;

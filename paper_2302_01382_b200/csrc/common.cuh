@@ -121,6 +121,8 @@ struct GemmArgs {
   const float* residual; int64_t ldr;  // optional fp32 addend (before act)
   int32_t* acc;                 // optional raw accumulators (int8 only) [m x n]
   CodeSlot slots[kMaxSlots];
+  float* amax = nullptr;        // optional: max |output| (after shortcut and activation) is folded into *amax, which
+                                // the caller has set to zero (calibration: the range of the consumers' input)
   // implicit-GEMM convolution (conv_kh > 0): `a` is the NHWC code tensor [batch*H*W x C] of the layer's
   // input (lda = C), m = batch*OH*OW, k = kh*kw*C; the kernel gathers the patches itself
   int conv_kh = 0, conv_kw = 0, conv_stride = 0, conv_pad = 0, conv_h = 0, conv_w = 0, conv_c = 0;

@@ -86,6 +86,7 @@ struct GroupDesc {
   float scale_x;
   const float* scale_w;
   const float* residual; int64_t ldr;
+  unsigned* amax;             // optional: bit pattern of max |output| over the whole matrix (general body only)
   OutDesc outs[kNumOuts];     // [0] raw accumulators, [1] fp32 output, [2..] consumer codes
 };
 // Implicit-GEMM convolution: the A operand is not a matrix in memory but the NHWC code tensor of the
@@ -616,6 +617,22 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
   } else if (p.act == QCFG_ACT_GELU_TANH) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) y[i] = gelu_tanh(y[i]);
+  }
+  if (p.amax) {     // calibration: the range of what the consumers will read (bit patterns, exact in any order)
+    unsigned mx = 0;
+    if (row_ok) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const unsigned a = __float_as_uint(y[i]) & 0x7fffffffu;
+        if (i < ncols) mx = mx > a ? mx : a;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned other = __shfl_xor_sync(0xffffffffu, mx, o);
+      mx = mx > other ? mx : other;
+    }
+    if (lane == 0 && mx) atomicMax(p.amax, mx);
   }
   if (p.outs[1].kind) {
     uint32_t w[32];
@@ -1526,9 +1543,10 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
     tn_total += (int32_t)((g.n + bn - 1) / bn);
     G.scale_x = g.scale_x; G.scale_w = g.scale_w; G.act = g.act;
     G.residual = g.residual; G.ldr = g.ldr;
+    G.amax = reinterpret_cast<unsigned*>(g.amax);
     if (g.acc && !g.is_bf16) { G.outs[0].kind = 4; G.outs[0].ptr = g.acc; G.outs[0].ld = g.n; }
     if (g.y) { G.outs[1].kind = 3; G.outs[1].ptr = g.y; G.outs[1].ld = g.ldy; }
-    G.need_y = g.y != nullptr;
+    G.need_y = g.y != nullptr || g.amax != nullptr;
     for (int s = 0; s < kMaxSlots; ++s) {
       if (!g.slots[s].kind) continue;
       OutDesc& o = G.outs[2 + s];
@@ -1543,7 +1561,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
     // staging per epilogue warp: two slots of 1 KB when only int8 codes are written, else of 2 KB
     for (int j = 0; j < kNumOuts; ++j) if (G.outs[j].kind >= 2 && G.outs[j].tma) wide = true;
     G.mode = EPI_GENERAL;
-    if (bn == 256 && !G.residual && !G.outs[0].kind && !G.outs[3].kind && !G.outs[4].kind) {
+    if (bn == 256 && !G.residual && !G.amax && !G.outs[0].kind && !G.outs[3].kind && !G.outs[4].kind) {
       if (!G.outs[1].kind && G.outs[2].kind == 1 && make_fast_map(&maps[i * kMapsPerGroup + MAP_FAST], G.outs[2], g.m, g.n)) G.mode = EPI_CODES1;
       else if (G.outs[1].kind && !G.outs[2].kind && make_fast_map(&maps[i * kMapsPerGroup + MAP_FAST], G.outs[1], g.m, g.n)) { G.mode = EPI_Y; wide = true; }
     }

@@ -318,3 +318,28 @@ def test_chained_and_separate_launches_agree_bitwise(ctx, m):
     finally:
         ctx.set_gemm_chains(True)
         model.close()
+
+
+def test_calibration_maxima_do_not_depend_on_fusion_or_chaining(ctx):
+    """The calibration forward may take an activation's range in the epilogue of the GEMM that
+    produces it (fusion on: the 16-bit operand codes come from there too, and the GEMMs chain) or in
+    the kernel that builds the 16-bit operand (fusion off).  Both read the same fp32 values and fold
+    bit patterns with an integer maximum, so the tables agree bit for bit."""
+    w = wl.bert_stack(5, 19200, 256, 1024, 2, bit_choices=None)
+    model, x = build(ctx, w)
+    try:
+        tables = {}
+        for fuse in (True, False):
+            for chained in (True, False):
+                ctx.set_fusion(fuse)
+                ctx.set_gemm_chains(chained)
+                model.calibrate_model(x, w.m)
+                tables[(fuse, chained)] = np.array(model.act_absmax(), np.float32)
+        ref = tables[(False, False)]
+        assert np.all(ref > 0)
+        for key, t in tables.items():
+            np.testing.assert_array_equal(t.view(np.uint32), ref.view(np.uint32), err_msg=str(key))
+    finally:
+        ctx.set_fusion(True)
+        ctx.set_gemm_chains(True)
+        model.close()
