@@ -115,6 +115,7 @@ int* pair_cluster_cache(Ctx* ctx) { return ctx->pair_clusters; }
 int device_of(Ctx* ctx) { return ctx->device; }
 void*& chain_slot(Ctx* ctx) { return ctx->chain_state; }
 bool ctx_chain_enabled(Ctx* ctx) { return ctx->chain != 0; }
+void ctx_disable_chains(Ctx* ctx) { ctx->chain = 0; }
 int prof_mode(Ctx* ctx) { return ctx->prof; }
 
 int set_error(Ctx* ctx, int code, const char* fmt, ...) {

@@ -25,6 +25,7 @@ int* pair_cluster_cache(Ctx* ctx);   // [2]: resident CTA pairs of the int8 / bf
 int device_of(Ctx* ctx);
 void*& chain_slot(Ctx* ctx);         // gemm.cu's per-context state
 bool ctx_chain_enabled(Ctx* ctx);
+void ctx_disable_chains(Ctx* ctx);
 int prof_mode(Ctx* ctx);
 // grows (never shrinks) the context's scratch buffer; returns nullptr on failure
 void* scratch(Ctx* ctx, size_t bytes);

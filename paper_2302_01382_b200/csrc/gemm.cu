@@ -1434,6 +1434,29 @@ int gemm_chain_flush(Ctx* ctx) {
   const cudaError_t le = cs->bf16 ? cudaLaunchKernelEx(&cfg, gemm_kernel<true, true, true, true>, A)
                                   : cudaLaunchKernelEx(&cfg, gemm_kernel<false, true, true, true>, A);
   A.n = 0;
+  if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorNotSupported) {
+    // The device cannot keep the whole grid resident right now (or does not take cooperative
+    // launches): nothing ran.  The records go out one by one through the ordinary flavour, in
+    // their order, and this context stops chaining.
+    (void)cudaGetLastError();
+    ctx_disable_chains(ctx);
+    cudaLaunchConfig_t one = cfg;
+    one.blockDim = dim3(kGemmThreads);
+    one.numAttrs = 2;
+    for (int i = 0; i < n; ++i) {
+      memset(&cs->solo, 0, sizeof(cs->solo));
+      memcpy(cs->solo.rec[0].m, A.rec[i].m, sizeof(A.rec[i].m));     // pool indices stay valid in the larger pool
+      cs->solo.rec[0].p = A.rec[i].p;
+      for (int d = 0; d < kMaxDeps; ++d) cs->solo.rec[0].p.deps[d] = -1;
+      cs->solo.n = 1;
+      cs->solo.total_tiles = A.rec[i].p.tiles_m * A.rec[i].p.tiles_n;
+      const cudaError_t se = cs->bf16 ? cudaLaunchKernelEx(&one, gemm_kernel<true, true, true, false>, cs->solo)
+                                      : cudaLaunchKernelEx(&one, gemm_kernel<false, true, true, false>, cs->solo);
+      if (se != cudaSuccess) return check_cuda(ctx, se, "gemm launch");
+      count_launch(ctx);
+    }
+    return check_cuda(ctx, cudaGetLastError(), "gemm launch");
+  }
   if (le != cudaSuccess) return check_cuda(ctx, le, "gemm chain launch");
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "gemm chain launch");
@@ -1588,7 +1611,7 @@ int launch_gemm_group(Ctx* ctx, const GemmArgs* gs_in, int count, cudaStream_t s
   ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
   // (a GEMM with fewer tiles than CTA pairs has nothing to overlap with: the wait for its
   // producer's rows would cost more than the launch boundary it saves)
-  const bool chainable = cs && cs->open && pair && !conv && bn == 256 && prof_mode(ctx) != 1 && p.tiles_m <= kChainMaxTilesM &&
+  const bool chainable = cs && cs->open && ctx_chain_enabled(ctx) && pair && !conv && bn == 256 && prof_mode(ctx) != 1 && p.tiles_m <= kChainMaxTilesM &&
                          2 * p.tiles_m * p.tiles_n >= sm_count(ctx);
   p.epi_bytes = (wide || chainable) ? 4096 : 2048;
   int stages = (kSmemMax - kSmemHeader - kCsBytes - 1024 - kEpiWarps * p.epi_bytes) / stage_bytes;
