@@ -165,3 +165,40 @@ def test_resnet50_batch128_sampled_images(ctx):
                 del qx, acc
             np.testing.assert_array_equal(outs[l].view(np.uint32), y_ref.view(np.uint32), err_msg=f"layer {l} image {img}")
     model.close()
+
+
+def test_bench_launch_configuration_gives_the_checked_outputs(ctx):
+    """bench.py asks for the last layer's output only, so most layers write nothing but their
+    consumers' codes (fast epilogue bodies) and the GEMMs go out as chains.  The teacher-forced
+    checks above ask for every layer's output.  Here the two meet: for configurations of the greedy
+    pass and one with 16-bit layers, the last layer's output of the benchmark's configuration (chains
+    on and off) equals, bit for bit, the one of the every-output evaluation."""
+    w = wl.bert_base_x12()
+    model, x, weights = build(ctx, w)
+    n = len(w.layers)
+    rank = np.arange(n)
+    seq = wl.greedy_sequence(rank, w.accept)
+    mixed = np.array([16 if i % 7 == 3 else (4 if i % 3 == 0 else 8) for i in range(n)], dtype=np.uint8)
+    last = torch.empty((w.m, w.layers[-1].n_out), device="cuda")
+    try:
+        for bits in (seq[0], seq[40], seq[71], mixed):
+            ys = [torch.full((w.m, lay.n_out), float("nan"), device="cuda") for lay in w.layers]
+            model.eval_config(bits, x, w.m, ys)
+            ctx.check_sync()
+            ref = ys[-1].cpu().numpy()
+            del ys
+            assert np.all(np.isfinite(ref))
+            for chained in (True, False):
+                ctx.set_gemm_chains(chained)
+                last.fill_(float("nan"))
+                n0 = ctx.launch_count()
+                model.eval_config(bits, x, w.m, [None] * (n - 1) + [last])
+                ctx.check_sync()
+                launches = ctx.launch_count() - n0
+                np.testing.assert_array_equal(last.cpu().numpy().view(np.uint32), ref.view(np.uint32),
+                                              err_msg=f"chains {chained}")
+                if chained and not np.any(np.asarray(bits) == 16):
+                    assert launches <= 5, launches          # one input quantization and three chains
+    finally:
+        ctx.set_gemm_chains(True)
+        model.close()
