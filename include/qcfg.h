@@ -76,10 +76,11 @@ int qcfg_destroy(qcfg_ctx* ctx);
 /* Synchronises `stream`, then returns and clears the device error word:
  * QCFG_OK, QCFG_ETIMEOUT, QCFG_ENONFINITE or QCFG_ECUDA.                                  */
 int qcfg_sync_status(qcfg_ctx* ctx, void* stream);
-/* Self-test of the failure path of the kernels' bounded waits (every device-side wait on a
- * barrier gives up after a time limit instead of hanging): enqueues a one-thread kernel that
- * waits on a barrier nothing arrives on, with a limit of limit_ns nanoseconds (1 .. 1e8).  The
- * wait runs out, the kernel sets the time-out bit of the context's error word and ends normally;
+/* Self-test of the failure path of the kernels' bounded waits (every device-side wait, on a
+ * barrier or on a counter in shared or global memory, gives up after a time limit instead of
+ * hanging): enqueues a one-warp kernel that runs each kind of wait once on something nothing
+ * ever signals, with a limit of limit_ns nanoseconds (1 .. 1e8) each.  Every wait has to run
+ * out; then the kernel sets the time-out bit of the context's error word and ends normally;
  * the next qcfg_sync_status returns QCFG_ETIMEOUT and clears it.  Nothing else is touched.   */
 int qcfg_selftest_wait_timeout(qcfg_ctx* ctx, uint64_t limit_ns, void* stream);
 /* Library-owned, NUL-terminated description of the last non-OK status of this context.   */

@@ -171,7 +171,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // Chains: waits until a counter of finished tiles has reached `need`.  Bounded like every other wait.
-__device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, volatile int* abort_flag, unsigned* err) {
+__device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, volatile int* abort_flag, unsigned* err,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   uint64_t t0 = 0;
   for (uint32_t it = 1;; ++it) {
     uint32_t v;
@@ -182,7 +183,7 @@ __device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, v
       if (*abort_flag) return false;
       const uint64_t now = global_timer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         atomicOr(err, ERR_TIMEOUT);
         *abort_flag = 1;
         return false;
@@ -192,7 +193,8 @@ __device__ __forceinline__ bool flag_wait(const unsigned* flag, uint32_t need, v
 }
 
 // Chains: waits until the CTA's dependency warp has cleared `need` tiles (a counter in shared memory).
-__device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volatile int* abort_flag, unsigned* err) {
+__device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volatile int* abort_flag, unsigned* err,
+                                             uint64_t limit_ns = kWaitLimitNs) {
   uint64_t t0 = 0;
   for (uint32_t it = 1;; ++it) {
     uint32_t v;
@@ -203,7 +205,7 @@ __device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volat
       if (*abort_flag) return false;
       const uint64_t now = global_timer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         atomicOr(err, ERR_TIMEOUT);
         *abort_flag = 1;
         return false;
@@ -213,7 +215,8 @@ __device__ __forceinline__ bool cleared_wait(uint32_t addr, uint32_t need, volat
 }
 
 // Chains: waits (whole warp) until every epilogue warp has reported `need` tiles; lane w reads warp w's counter.
-__device__ __forceinline__ bool reported_wait(uint32_t rep0, uint32_t need, int lane, volatile int* abort_flag, unsigned* err) {
+__device__ __forceinline__ bool reported_wait(uint32_t rep0, uint32_t need, int lane, volatile int* abort_flag, unsigned* err,
+                                              uint64_t limit_ns = kWaitLimitNs) {
   uint64_t t0 = 0;
   for (uint32_t it = 1;; ++it) {
     uint32_t v = need;
@@ -224,7 +227,7 @@ __device__ __forceinline__ bool reported_wait(uint32_t rep0, uint32_t need, int 
       bool give_up = *abort_flag != 0;
       const uint64_t now = global_timer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         if (lane == 0) { atomicOr(err, ERR_TIMEOUT); *abort_flag = 1; }
         give_up = true;
       }
@@ -1204,6 +1207,7 @@ struct ChainState {
   ChainRecInfo info[kChainMax];
   double ops = 0.0;
   unsigned* ring = nullptr;       // device counters, handed out front to back and cleared when used up
+  unsigned* zero = nullptr;       // a device word that stays zero (self-test of the bounded waits)
   size_t ring_used = 0;           // bytes
   bool open = false;              // a forward pass is running: eligible launches may be deferred
   bool bf16 = false;
@@ -1297,24 +1301,43 @@ bool make_fast_map(CUtensorMap* map, const OutDesc& o, int64_t m, int64_t n) {
                    CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
-// Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on, with
-// a caller-chosen limit; the wait gives up, sets the time-out bit of the error word and the
-// kernel ends normally.
-__global__ void wait_timeout_kernel(uint64_t limit_ns, unsigned* err) {
+// Self-test of the bounded waits: the kernel waits on a barrier nothing ever arrives on and on
+// counters (global and shared) nothing ever advances, each with a caller-chosen limit.  Every wait
+// has to give up; only then does the last one set the time-out bit of the error word.  The kernel
+// ends normally either way.
+__global__ void wait_timeout_kernel(uint64_t limit_ns, unsigned* err, const unsigned* zero_word) {
   __shared__ uint64_t bar;
   __shared__ int abort_flag;
+  __shared__ unsigned local_err;
+  __shared__ uint32_t counters[kEpiWarps + 1];
   if (threadIdx.x == 0) {
     abort_flag = 0;
+    local_err = 0;
+    for (int i = 0; i <= kEpiWarps; ++i) counters[i] = 0;
     mbar_init(smem_u32(&bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    (void)mbar_wait(smem_u32(&bar), 0, &abort_flag, err, limit_ns);
+  }
+  __syncwarp();
+  const int lane = threadIdx.x & 31;
+  // whole-warp wait on the per-warp report counters
+  const bool gave_up_rep = !reported_wait(smem_u32(&counters[0]), 1u, lane, &abort_flag, &local_err, limit_ns);
+  bool all = gave_up_rep;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    all = all && !cleared_wait(smem_u32(&counters[kEpiWarps]), 1u, &abort_flag, &local_err, limit_ns);
+    abort_flag = 0;
+    all = all && !flag_wait(zero_word, 1u, &abort_flag, &local_err, limit_ns);
+    abort_flag = 0;
+    if (all) (void)mbar_wait(smem_u32(&bar), 0, &abort_flag, err, limit_ns);
   }
 }
 
 }  // namespace
 
 int launch_wait_timeout(Ctx* ctx, uint64_t limit_ns, cudaStream_t st) {
-  wait_timeout_kernel<<<1, 32, 0, st>>>(limit_ns, err_word(ctx));
+  ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
+  if (!cs) return set_error(ctx, QCFG_ESTATE, "wait self-test: context not initialised");
+  wait_timeout_kernel<<<1, 32, 0, st>>>(limit_ns, err_word(ctx), cs->zero);
   count_launch(ctx);
   return check_cuda(ctx, cudaGetLastError(), "wait self-test launch");
 }
@@ -1342,7 +1365,14 @@ int gemm_init(Ctx* ctx) {
   if (!cs) return set_error(ctx, QCFG_ENOMEM, "gemm: host allocation failed");
   e = cudaMalloc(&cs->ring, kFlagRingBytes);
   if (e == cudaSuccess) e = cudaMemset(cs->ring, 0, kFlagRingBytes);
-  if (e != cudaSuccess) { delete cs; return check_cuda(ctx, e, "gemm chain counters"); }
+  if (e == cudaSuccess) e = cudaMalloc(&cs->zero, sizeof(unsigned));
+  if (e == cudaSuccess) e = cudaMemset(cs->zero, 0, sizeof(unsigned));
+  if (e != cudaSuccess) {
+    if (cs->ring) cudaFree(cs->ring);
+    if (cs->zero) cudaFree(cs->zero);
+    delete cs;
+    return check_cuda(ctx, e, "gemm chain counters");
+  }
   chain_slot(ctx) = cs;
   return QCFG_OK;
 }
@@ -1351,6 +1381,7 @@ void gemm_destroy(Ctx* ctx) {
   ChainState* cs = static_cast<ChainState*>(chain_slot(ctx));
   if (!cs) return;
   if (cs->ring) cudaFree(cs->ring);
+  if (cs->zero) cudaFree(cs->zero);
   delete cs;
   chain_slot(ctx) = nullptr;
 }

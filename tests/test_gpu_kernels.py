@@ -299,8 +299,10 @@ def test_argument_errors_leave_outputs_untouched(ctx):
 # ----------------------------------------------------------------------------- device-side faults
 
 def test_bounded_wait_gives_up_and_the_context_stays_usable(ctx):
-    """A device wait whose barrier is never signalled runs into its limit (1 ms here), reports
-    QCFG_ETIMEOUT through the error word, and leaves the context able to run a correct GEMM."""
+    """Device waits on a barrier that is never signalled and on counters that never advance (the
+    waits of the chained GEMM launches) each run into their limit (1 ms here); only when all of
+    them gave up does the kernel report QCFG_ETIMEOUT through the error word.  The context is left
+    able to run a correct GEMM."""
     import paper_2302_01382_b200 as q
     assert ctx.sync_status() == q.OK
     ctx.selftest_wait_timeout(1_000_000)
