@@ -673,8 +673,9 @@ __device__ __forceinline__ void epilogue_chunk(const GroupDesc& p, const CUtenso
 // CTA pairs deal out round-robin, so a pair that runs out of tiles of one record goes on with the
 // next: no pipeline fill and drain, no idle last round and no kernel boundary between layers.
 // A tile may start when the row tiles it reads are complete: every finished tile adds one to a
-// counter of its (record, row tile, CTA rank), a warp of its own does that once the tile's stores
-// have completed, and the producer warp waits for the counters of the records its record names.
+// counter of its (record, row tile, CTA rank) -- a warp of its own does that once the tile's stores
+// have completed -- and another warp, ahead of the producer, waits for the counters of the records
+// a tile's record names and clears the tile for loading.
 // Waits only ever point at earlier tiles of the sequence and the launch is cooperative (all CTAs
 // resident), so the first unfinished tile can always proceed.  The records of a chain share tile
 // shape, operand type, stage count, staging size, rows and grid.
